@@ -122,6 +122,17 @@ def executed_units(plan, w):
     return total
 
 
+def listed_pair_flops(plan, w):
+    """4*d * sum over (query block, listed KV block) of BS*BS: what the lists ask for with every block padded
+    to its nominal size, before 64-token query blocks are paired into 128-row tiles."""
+    t = plan.tables()
+    total = 0.0
+    for bh, c in enumerate(t["scheme"].cpu().tolist()):
+        g = plan.geometry(c)
+        total += float(t["kv_cnt"][bh, :g["NB"]].sum()) * g["BS"] * g["BS"]
+    return 4.0 * w.d * total
+
+
 def achieved_sparsity(plan, w):
     """1 - kept token pairs / N^2 (fraction of pruned attention scores), from the GPU's lists."""
     t = plan.tables()
@@ -176,24 +187,47 @@ def oracle_sample_seconds(w, forced, Qb, Kb, Vb, n_blocks=4, threads=0):
     return total, desc, cores
 
 
+def _config(w, forced, args, **extra):
+    """The `config` object both arms print (same keys, so the two lines can be matched)."""
+    cfg = dict(workload=w.name, heads=w.heads, grid=list(w.grid), n_text=w.n_text, N=w.n_tokens, d=w.d,
+               candidates=[list(c) for c in w.candidates], mode=w.mode, budget=w.value,
+               forced_scheme=None if forced is None else forced[0], amplitude=w.amplitude,
+               static_masks=dict(window=args.window, sink_tokens=args.sink, intra_threshold=args.intra),
+               estimator=args.estimator)
+    cfg.update(extra)
+    return cfg
+
+
 def run_reference(args, w, forced):
-    """`--impl reference`: the oracle, as it stands, on the host cores (rank 0 only)."""
+    """`--impl reference`: the oracle, as it stands, on the host cores (rank 0 only).  Each step is a bounded
+    sample of the workload (head 0: selection in full, attention on 16 query blocks); the printed
+    ms_per_step is that sample's time scaled to all blocks and heads, and says so."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    Q, K, V = make_qkv(w, "cpu", heads=[0])
-    Qb, Kb, Vb = (bf16_bits(x)[0] for x in (Q, K, V))
-    times = []
+    # the same generator stream as the GPU arm when a device is there (so head 0 holds the same bytes);
+    # torch's CPU stream of the same seed otherwise
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    Q, K, V = make_qkv(w, gen_dev, heads=[0])
+    Qb, Kb, Vb = (bf16_bits(x[:, :1])[0] for x in (Q, K, V))
+    del Q, K, V
+    times, sample_s = [], []
     desc, cores = "", 1
     for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
         sec, desc, cores = oracle_sample_seconds(w, forced, Qb, Kb, Vb, n_blocks=16)
         if i >= args.warmup:
             times.append(sec)
+            sample_s.append(time.perf_counter() - t0)
     sec = sum(times) / len(times)
     val = w.dense_flops() / sec / 1e12
     line = dict(impl="reference", metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
-                warmup=args.warmup, ms_per_step=sec * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
-                dtype="f64", data="synthetic", config=dict(workload=w.name, sample=desc),
-                cpu_baseline=dict(value=val, unit=UNIT, cores=cores, kind="oracle", sample=desc),
+                warmup=args.warmup, ms_per_step=sec * 1e3, extrapolated=True,
+                measured_sample_ms_per_step=sum(sample_s) / len(sample_s) * 1e3,
+                higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic",
+                config=_config(w, forced, args, sample=desc,
+                               generator=f"torch {gen_dev} generator streams of seed {w.seed} (head 0 only)"),
+                cpu_baseline=dict(value=val, unit=UNIT, cores=cores, kind="oracle", sample=desc, extrapolated=True),
                 e2e=dict(value=val, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line))
 
@@ -201,10 +235,11 @@ def run_reference(args, w, forced):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="wan1p3b")
+    ap.add_argument("--workload", default="wan14b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--heads", type=int, default=0, help="run a slice of the workload with this many heads (profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--window", type=int, default=-1, help="local-window radius in blocks (static mask), < 0 = off")
@@ -215,6 +250,8 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w, forced = _workload(args.workload)
+    if args.heads > 0:
+        w = w.replace(name=f"{w.name}_heads{args.heads}", heads=args.heads)
     if forced is not None:
         forced = forced * (w.heads * w.batch)
 
@@ -281,25 +318,50 @@ def main():
     peaks = _peaks()
     units = executed_units(plan, w)
     exec_flops = 4.0 * w.d * units * 128 * 64
+    listed_flops = listed_pair_flops(plan, w)
     attn_ms = stage_ms[3]
     achieved = exec_flops / (attn_ms * 1e-3) / 1e12
+    sparsity = achieved_sparsity(plan, w)
+    useful_flops = (1.0 - sparsity) * w.dense_flops()
+    useful = useful_flops / (attn_ms * 1e-3) / 1e12
+    # DRAM traffic of one launch: only from an ncu capture of this very workload (profiles/), else null
     traffic = None
     prof = os.path.join(ROOT, "profiles", f"k_attn_{w.name}.txt")
     if os.path.exists(prof):
         for ln in open(prof):
             if ln.startswith("dram_bytes_per_launch:"):
                 traffic = float(ln.split(":")[1].split()[0])
-    sel_bytes = 2.0 * w.heads * w.batch * w.n_tokens * w.d * 2
-    roofline = dict(bound="tensor", kernel="k_attn", achieved=achieved, peak=peaks["bf16_sustained"], unit="TFLOP/s",
-                    frac=achieved / peaks["bf16_sustained"], frac_of_burst_peak=achieved / peaks["bf16"],
-                    peak_kind="bf16 sustained, " + peaks["kind"], traffic=traffic,
-                    executed_tflop_per_launch=exec_flops / 1e12, launch_ms=attn_ms)
-    sparsity = achieved_sparsity(plan, w)
-    stages = dict(achieved_sparsity=sparsity, useful_tflops=(1.0 - sparsity) * w.dense_flops() / (attn_ms * 1e-3) / 1e12,
+    # Which measured peak the run compares with follows from the run: the burst figure when the timed region
+    # is short or the clocks stayed at their maximum without the power cap, the sustained one otherwise.
+    sm, smax = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    at_max = sm is not None and smax is not None and sm >= 0.985 * smax and "sw_power_cap" not in clocks.get("reasons", [])
+    burst = total_ms < 1000.0 or at_max
+    peak = peaks["bf16"] if burst else peaks["bf16_sustained"]
+    roofline = dict(bound="tensor", kernel="k_attn", achieved=achieved, peak=peak, unit="TFLOP/s",
+                    frac=achieved / peak, peak_kind=("bf16 burst, " if burst else "bf16 sustained, ") + peaks["kind"],
+                    frac_of_burst_peak=achieved / peaks["bf16"], frac_of_sustained_peak=achieved / peaks["bf16_sustained"],
+                    useful_frac=useful / peak, traffic=traffic,
+                    executed_tflop_per_launch=exec_flops / 1e12, launch_ms=attn_ms,
+                    launch_ms_x_sm_mhz=None if sm is None else attn_ms * sm,
+                    algorithmic_dram_bytes_per_launch=4.0 * w.heads * w.batch * w.n_tokens * w.d * 2)
+    # selection stages (plan + summarize + select): algorithmic bytes = Q and K read once, the chosen
+    # scheme's summaries and the index lists written once
+    t_tab = plan.tables()
+    list_bytes = 4.0 * float(t_tab["kv_cnt"].sum())
+    summ_bytes = 2.0 * 512.0 * sum(plan.geometry(c)["NB"] for c in t_tab["scheme"].cpu().tolist())
+    qk_bytes = 2.0 * w.heads * w.batch * w.n_tokens * w.d * 2
+    sel_bytes = qk_bytes + summ_bytes + list_bytes
+    sel_ms = stage_ms[0] + stage_ms[1] + stage_ms[2]
+    stages = dict(achieved_sparsity=sparsity, useful_tflops=useful,
+                  executed_split=dict(valid_token_pairs=useful_flops / exec_flops,
+                                      edge_padding_of_listed_blocks=(listed_flops - useful_flops) / exec_flops,
+                                      unlisted_half_of_paired_tiles=(exec_flops - listed_flops) / exec_flops),
                   plan_ms=stage_ms[0], summarize_ms=stage_ms[1], select_ms=stage_ms[2], attn_ms=stage_ms[3],
-                  selection_hbm_gbs=sel_bytes / ((stage_ms[0] + stage_ms[1] + stage_ms[2]) * 1e-3) / 1e9,
-                  selection_hbm_frac=sel_bytes / ((stage_ms[0] + stage_ms[1] + stage_ms[2]) * 1e-3) / 1e9 / peaks["hbm"],
-                  summarize_hbm_gbs=sel_bytes / (stage_ms[1] * 1e-3) / 1e9)
+                  plan_summarize_hbm_gbs=(qk_bytes + summ_bytes) / ((stage_ms[0] + stage_ms[1]) * 1e-3) / 1e9,
+                  selection_ms=sel_ms, selection_algorithmic_bytes=sel_bytes,
+                  selection_hbm_gbs=sel_bytes / (sel_ms * 1e-3) / 1e9,
+                  selection_hbm_frac=sel_bytes / (sel_ms * 1e-3) / 1e9 / peaks["hbm"],
+                  hbm_peak_gbs=peaks["hbm"])
 
     t = plan.tables()
     schemes_chosen = t["group_count"].cpu().tolist()[:len(w.candidates)]
@@ -336,16 +398,14 @@ def main():
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                     ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
                     data="synthetic",
-                    config=dict(workload=w.name, heads=w.heads, grid=list(w.grid), n_text=w.n_text, N=w.n_tokens, d=w.d,
-                                candidates=[list(c) for c in w.candidates], mode=w.mode, budget=w.value,
-                                forced_scheme=None if forced is None else forced[0], amplitude=w.amplitude,
-                                static_masks=dict(window=args.window, sink_tokens=args.sink, intra_threshold=args.intra),
-                                estimator=args.estimator,
-                                l2="inputs larger than L2 (Q+K+V+O = %.0f MB)" % (4 * nbytes / 1e6),
-                                schemes_chosen=schemes_chosen, pairing_axes=pairing_axes),
+                    config=_config(w, forced, args, l2="inputs larger than L2 (Q+K+V+O = %.0f MB)" % (4 * nbytes / 1e6),
+                                   schemes_chosen=schemes_chosen, pairing_axes=pairing_axes),
                     roofline=roofline, stages=stages, cpu_baseline=cpu, e2e=e2e, clocks=clocks,
                     gpu_launches=args.steps * kernel_launches,
-                    executed_tflops=achieved, useful_note="executed = 128x64 units as multiplied (padding and merged lists included)")
+                    executed_tflops=achieved,
+                    useful_note="executed = 128x64 units as multiplied; executed_split says how much of it is valid token "
+                                "pairs, zero-filled edge padding of listed blocks, and the half of a paired 64-token tile "
+                                "that does not list the unit")
         print(json.dumps(line))
     plan.close()
     if dist is not None:

@@ -27,8 +27,13 @@
  *     by spade_plan_destroy).  A plan and a workspace serve one layer at a time: calls on the same
  *     plan must not overlap in time (host threads) and a workspace must not be used by two layers
  *     that may run concurrently (streams); use one plan and one workspace per concurrent layer.
+ *     The attention and estimator kernels take their tensor-memory columns with tcgen05.alloc, the one
+ *     device-side wait of this library that has no time limit (the instruction has none): two layers
+ *     launched on two streams are correct but take turns on an SM's tensor memory rather than overlap.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Stage calls are
- *     asynchronous and never synchronise the host.
+ *     asynchronous and never synchronise the host.  Every call makes the plan's device current
+ *     while it runs and restores the caller's current device before it returns.
+ *   - B * heads may be at most 4096.
  *   - Every function returns SPADE_OK (0) or a negative spade_error_t; arguments are validated
  *     before anything is launched; nothing aborts.  spade_last_error() gives the message.
  *   - There is no CPU path: without a CUDA device every stage returns SPADE_ERR_CUDA.
@@ -46,7 +51,7 @@ extern "C" {
 typedef enum {
   SPADE_OK = 0,
   SPADE_ERR_INVALID_ARG = -1,     /* null pointer, non-positive size, bad mode / value, misaligned pointer */
-  SPADE_ERR_UNSUPPORTED = -2,     /* d != 128, block size not in {64,128}, more than 2048 blocks, > 8 candidates */
+  SPADE_ERR_UNSUPPORTED = -2,     /* d != 128, block size not in {64,128}, more than 2048 blocks, > 8 candidates, B*heads > 4096 */
   SPADE_ERR_WORKSPACE = -3,       /* workspace pointer null or misaligned */
   SPADE_ERR_CUDA = -4,            /* a CUDA runtime / driver call failed (message holds the CUDA error) */
   SPADE_ERR_DEVICE_TIMEOUT = -5,  /* a bounded device-side wait ran out (reported by spade_status) */
@@ -116,7 +121,9 @@ size_t spade_workspace_bytes(const spade_plan_t* plan);
 
 /* Stage 1 (Eq. 3-5, Algorithm 1; Sec. 3.2).  forced_scheme: optional HOST array of B*heads
  * candidate indices; if non-NULL the Aggregation Scores are not computed and each head takes
- * the given candidate (the array is copied before the call returns). */
+ * the given candidate.  The array is read before the call returns and never afterwards, pinned or
+ * not: the schemes travel as an argument of the launch, so a launch captured in a CUDA graph replays
+ * the schemes it was captured with. */
 int spade_plan(spade_plan_t* plan, const void* Q, const void* K, void* ws, void* stream, const int32_t* forced_scheme);
 /* Stage 2 (Sec. 3.1, 3.3).  Needs spade_plan on the same workspace first. */
 int spade_summarize(spade_plan_t* plan, const void* Q, const void* K, void* ws, void* stream);
@@ -194,10 +201,12 @@ int spade_launch_count(const spade_plan_t* plan);
  * Some code that wants the per-candidate Aggregation Scores cannot obtain device memory at the
  * moment it runs: a plugin living inside another framework whose caching allocator owns the whole
  * device, a service with a fixed, pre-reserved memory budget, or a latency-critical loop where a
- * cudaMalloc (which may synchronise the device) is off the table.  For them this call computes the
- * same numbers as spade_plan's `as` table -- AS(Q|c) and AS(K|c) for every head and candidate --
- * but needs no workspace: the per-block SICS values, which the other path keeps in the caller's
- * workspace, go to a fixed array that is part of the library image itself.
+ * cudaMalloc (which may synchronise the device) is off the table.  For them this call computes what
+ * spade_plan leaves in its `as` table -- AS(Q|c) and AS(K|c) for every head and candidate -- but
+ * needs no workspace: the per-block SICS values, which the other path keeps in the caller's
+ * workspace, go to a fixed array that is part of the library image itself.  The two entry points
+ * agree to fp32 rounding, not bit for bit: this one always reduces each block from its token rows,
+ * spade_plan usually adds up per-cell sums shared by all candidates, a different summation order.
  *
  *   as_out   DEVICE pointer, float [B*heads][n_cands][2] (Q then K), written by the call.
  *   Q, K     as for spade_plan.
@@ -207,7 +216,12 @@ int spade_launch_count(const spade_plan_t* plan);
  * nothing is launched.  Every GPU that loads the library carries those 4 MiB until the process exits.
  * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.  The first
  * call on a device looks up the array's device address (once per device, with that device
- * current); make that first call outside any stream capture.  All calls on one device share the
+ * current); make that first call outside any stream capture.  That look-up is also the moment the
+ * CUDA runtime loads this library's device code on that GPU, the 4 MiB included, if nothing of the
+ * library ran there before: on a device another allocator has filled to the brim this is where
+ * SPADE_ERR_CUDA (out of memory) can still come from, so make the first call at start-up.  The
+ * address is remembered for the life of the device's primary context; after cudaDeviceReset the
+ * process must not call this entry point again.  All calls on one device share the
  * array and it keeps whatever the previous call left in it; every value a call reads it has
  * written itself first, so nothing has to be cleared -- but two calls whose kernels overlap in
  * time on the same GPU (different streams, different plans, different threads) race on it:

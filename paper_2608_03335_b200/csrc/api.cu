@@ -31,6 +31,20 @@ int fail(int code, const char* fmt, ...) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Makes the plan's device current for the duration of a call and puts the caller's device back.
+struct DeviceGuard {
+  int prev = -1, want = -1;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceGuard(int device) : want(device) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != device) err = cudaSetDevice(device);
+  }
+  ~DeviceGuard() { if (prev >= 0 && prev != want) cudaSetDevice(prev); }
+};
+#define ON_PLAN_DEVICE(p)              \
+  DeviceGuard guard__((p)->device);    \
+  CUDA_TRY(guard__.err)
+
 struct WsLayout {
   size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, scores, colkeep, rowfull, pair_axis, pair_union, mm, text_start, head_work, att_scratch;
   size_t bytes;
@@ -45,8 +59,7 @@ struct spade_plan_s {
   Shape sh;
   GeoPack gp;
   StaticTables st;
-  void* d_static;        // one allocation holding rowoff, nvalid, kvalid, budget, forced
-  int* d_forced;
+  void* d_static;        // one allocation holding rowoff, nvalid, kvalid, budget
   WsLayout lay;
   ScoreMaps* smaps;      // tensor map of the K' summaries inside `smaps_ws`
   const void* smaps_ws;
@@ -181,7 +194,8 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
     return fail(SPADE_ERR_INVALID_ARG, "bad grid %dx%dx%d + %d text", grid->T, grid->H, grid->W, grid->n_text);
   if (n_cands < 1) return fail(SPADE_ERR_INVALID_ARG, "n_cands must be at least 1");
   if (n_cands > SPADE_MAX_CANDS) return fail(SPADE_ERR_UNSUPPORTED, "more than %d candidates", SPADE_MAX_CANDS);
-  if ((long)B * heads > 65535) return fail(SPADE_ERR_UNSUPPORTED, "B*heads above 65535");
+  // the head ordering of the plan and select stages ranks the heads pairwise in one CTA
+  if ((long)B * heads > SPADE_MAX_BH) return fail(SPADE_ERR_UNSUPPORTED, "B*heads above %d", SPADE_MAX_BH);
   if (budget->mode < 0 || budget->mode > 3) return fail(SPADE_ERR_INVALID_ARG, "unknown budget mode %d", budget->mode);
   const int BH = B * heads;
   for (int i = 0; i < BH; ++i) {
@@ -301,8 +315,7 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
   const size_t o_nvalid = align_up(o_rowoff + rowoff.size() * 4, 256);
   const size_t o_kvalid = align_up(o_nvalid + nvalid.size() * 4, 256);
   const size_t o_budget = align_up(o_kvalid + kvalid.size() * 8, 256);
-  const size_t o_forced = align_up(o_budget + bud.size() * 4, 256);
-  const size_t total = align_up(o_forced + (size_t)BH * 4, 256);
+  const size_t total = align_up(o_budget + bud.size() * 4, 256);
   e = cudaMalloc(&p->d_static, total);
   if (e != cudaSuccess) { free(p); return fail(SPADE_ERR_CUDA, "cudaMalloc(%zu): %s", total, cudaGetErrorString(e)); }
   char* base = (char*)p->d_static;
@@ -315,14 +328,16 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
   p->st.nvalid = (const int*)(base + o_nvalid);
   p->st.kvalid = (const uint64_t*)(base + o_kvalid);
   p->st.budget = (const float*)(base + o_budget);
-  p->d_forced = (int*)(base + o_forced);
 
   p->base_cap = sh.cap;
   compute_layout(p);
 
   p->maps = (AttnMaps*)calloc(1, attn_maps_bytes());
   p->smaps = (ScoreMaps*)calloc(1, score_maps_bytes());
-  if (!p->maps || !p->smaps) { cudaFree(p->d_static); free(p); return fail(SPADE_ERR_INVALID_ARG, "out of host memory"); }
+  if (!p->maps || !p->smaps) {
+    cudaFree(p->d_static); free(p->maps); free(p->smaps); free(p);
+    return fail(SPADE_ERR_INVALID_ARG, "out of host memory");
+  }
   *out = p;
   return SPADE_OK;
 }
@@ -405,12 +420,19 @@ int spade_plan(spade_plan_t* p, const void* Q, const void* K, void* ws, void* st
     for (int i = 0; i < p->sh.BH; ++i)
       if (forced[i] < 0 || forced[i] >= p->sh.C) return fail(SPADE_ERR_INVALID_ARG, "forced_scheme[%d] = %d out of range", i, forced[i]);
   cudaStream_t s = (cudaStream_t)stream;
-  CUDA_TRY(cudaSetDevice(p->device));
+  ON_PLAN_DEVICE(p);
   WsTables t = tables_at(p, ws);
   p->launches = 0;
   if (!p->keep_status) CUDA_TRY(cudaMemsetAsync(t.status, 0, 64 * 4, s));
   const bool skip_sics = forced != nullptr && !(p->sh.masks_on && p->sh.intra_thr > 0.f) && p->sh.mode != SPADE_POLICY_AS;
-  if (forced) CUDA_TRY(cudaMemcpyAsync(p->d_forced, forced, (size_t)p->sh.BH * 4, cudaMemcpyHostToDevice, s));
+  // The caller's array is read here and never again: the schemes travel inside the launch itself
+  // (4 bits per head), so a captured launch replays the values it was captured with.
+  ForcedPack fpack;
+  memset(&fpack, 0, sizeof(fpack));
+  if (forced) {
+    fpack.on = 1;
+    for (int i = 0; i < p->sh.BH; ++i) fpack.w[i >> 3] |= (uint32_t)forced[i] << ((i & 7) * 4);
+  }
   p->have_csum = 0;
   if (!skip_sics) {
     if (p->sh.use_cells) {
@@ -423,7 +445,7 @@ int spade_plan(spade_plan_t* p, const void* Q, const void* K, void* ws, void* st
       p->launches += 1;
     }
   }
-  CUDA_TRY(launch_choose(p->sh, p->gp, p->st, t, forced ? p->d_forced : nullptr, skip_sics ? 0 : 1, s));
+  CUDA_TRY(launch_choose(p->sh, p->gp, p->st, t, fpack, skip_sics ? 0 : 1, s));
   p->launches += 2;
   if (p->sh.masks_on) {
     CUDA_TRY(launch_static(p->sh, p->gp, p->st, t, s));
@@ -438,8 +460,8 @@ int spade_summarize(spade_plan_t* p, const void* Q, const void* K, void* ws, voi
   if (rc) return rc;
   if ((rc = check_tensor(Q, "Q")) || (rc = check_tensor(K, "K"))) return rc;
   if (p->stage < 1 || p->stage_ws != ws) return fail(SPADE_ERR_ORDER, "spade_summarize needs spade_plan on this workspace first");
-  CUDA_TRY(cudaSetDevice(p->device));
-  if (p->have_csum) CUDA_TRY(launch_gather(p->sh, p->gp, tables_at(p, ws), (cudaStream_t)stream));
+  ON_PLAN_DEVICE(p);
+  if (p->have_csum) CUDA_TRY(launch_gather(p->sh, p->gp, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
   else CUDA_TRY(launch_summarize(Q, K, p->sh, p->gp, p->st, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
   p->launches += 1;
   if (p->sh.estimator) {
@@ -454,7 +476,7 @@ int spade_select(spade_plan_t* p, void* ws, void* stream) {
   int rc = check_call(p, ws);
   if (rc) return rc;
   if (p->stage < 2 || p->stage_ws != ws) return fail(SPADE_ERR_ORDER, "spade_select needs spade_summarize on this workspace first");
-  CUDA_TRY(cudaSetDevice(p->device));
+  ON_PLAN_DEVICE(p);
   WsTables t = tables_at(p, ws);
   if (p->sh.estimator) {
     CUDA_TRY(launch_scores_minmax(p->sh, p->gp, t, (cudaStream_t)stream));
@@ -473,7 +495,7 @@ int spade_select(spade_plan_t* p, void* ws, void* stream) {
   if (any_pair) {
     // pair the 64-token query blocks along the axis that gives the shortest merged lists, per head
     CUDA_TRY(cudaMemsetAsync(t.pair_union, 0, (size_t)p->sh.BH * 3 * 4, (cudaStream_t)stream));
-    CUDA_TRY(launch_pair_axis(p->sh, p->gp, t, (cudaStream_t)stream));
+    CUDA_TRY(launch_pair_axis(p->sh, p->gp, t, p->num_sms, (cudaStream_t)stream));
     p->launches += 1;
   }
   CUDA_TRY(launch_groups_after_select(p->sh, p->gp, t, (cudaStream_t)stream));
@@ -487,7 +509,7 @@ int spade_attn(spade_plan_t* p, const void* Q, const void* K, const void* V, voi
   if (rc) return rc;
   if ((rc = check_tensor(Q, "Q")) || (rc = check_tensor(K, "K")) || (rc = check_tensor(V, "V")) || (rc = check_tensor(O, "O"))) return rc;
   if (p->stage < 1 || p->stage_ws != ws) return fail(SPADE_ERR_ORDER, "spade_attn needs spade_plan (and index lists) on this workspace first");
-  CUDA_TRY(cudaSetDevice(p->device));
+  ON_PLAN_DEVICE(p);
   if (Q != p->mq || K != p->mk || V != p->mv || O != p->mo) {
     char msg[256];
     if (attn_encode_maps(p->maps, Q, K, V, O, p->sh, p->gp, msg, sizeof(msg))) return fail(SPADE_ERR_CUDA, "tensor map: %s", msg);
@@ -517,7 +539,7 @@ int spade_forward_host(spade_plan_t* p, const void* hQ, const void* hK, const vo
   if (!p) return fail(SPADE_ERR_INVALID_ARG, "plan is NULL");
   if (!hQ || !hK || !hV || !hO) return fail(SPADE_ERR_INVALID_ARG, "a host tensor is NULL");
   cudaStream_t s = (cudaStream_t)stream;
-  CUDA_TRY(cudaSetDevice(p->device));
+  ON_PLAN_DEVICE(p);
   int rc;
   if ((rc = check_call(p, ws))) return rc;
   if ((rc = check_tensor(dQ, "dQ")) || (rc = check_tensor(dK, "dK")) || (rc = check_tensor(dV, "dV")) || (rc = check_tensor(dO, "dO"))) return rc;
@@ -558,7 +580,6 @@ int spade_forward_host(spade_plan_t* p, const void* hQ, const void* hK, const vo
     spade_plan_s view = *p;                           // shares the static tables and the descriptor scratch
     view.sh.BH = nh;
     view.st.budget = p->st.budget + h0;
-    view.d_forced = p->d_forced + h0;
     view.keep_status = g > 0;
     view.stage = 0; view.stage_ws = nullptr; view.smaps_ws = nullptr;
     view.mq = view.mk = view.mv = view.mo = nullptr;
@@ -589,7 +610,7 @@ int spade_forward_host(spade_plan_t* p, const void* hQ, const void* hK, const vo
 int spade_status(spade_plan_t* p, void* ws, void* stream) {
   int rc = check_call(p, ws);
   if (rc) return rc;
-  CUDA_TRY(cudaSetDevice(p->device));
+  ON_PLAN_DEVICE(p);
   uint32_t st[4] = {0, 0, 0, 0};
   CUDA_TRY(cudaMemcpyAsync(st, tables_at(p, ws).status, sizeof(st), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
   CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
@@ -625,8 +646,10 @@ constexpr int NOALLOC_MAX_DEVICES = 64;
 std::mutex g_noalloc_mutex;
 float* g_noalloc_ptr[NOALLOC_MAX_DEVICES];      // device address of the array, per device ordinal
 
-// AS(X|c) = sum of the per-block SICS (Eq. 3), added in the same fixed order the planning stage
-// uses (lane-strided partial sums, then a butterfly), so both entry points give identical bits.
+// AS(X|c) = sum of the per-block SICS (Eq. 3), added in the fixed order the planning stage uses
+// (lane-strided partial sums, then a butterfly).  The block values themselves come from the
+// per-candidate token pass here; the planning stage usually builds them from shared cell sums, so the
+// two entry points agree to fp32 summation order, not bit for bit.
 __global__ void __launch_bounds__(32)
 k_as_from_scratch(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp,
                   const float* __restrict__ sics, float* __restrict__ as_out) {
@@ -657,7 +680,7 @@ extern "C" int spade_aggregation_scores_noalloc(spade_plan_t* p, const void* Q, 
                 "holds %u -- use spade_plan with a workspace instead",
                 need, p->sh.BH, p->sh.C, p->sh.NBvmax, (unsigned)SPADE_NOALLOC_MAX_FLOATS);
   if (p->device < 0 || p->device >= NOALLOC_MAX_DEVICES) return fail(SPADE_ERR_UNSUPPORTED, "device ordinal %d", p->device);
-  CUDA_TRY(cudaSetDevice(p->device));
+  ON_PLAN_DEVICE(p);
   float* scratch;
   {
     // Once per device: in host code the array's name is only a handle, so ask the runtime for the
@@ -678,5 +701,6 @@ extern "C" int spade_aggregation_scores_noalloc(spade_plan_t* p, const void* Q, 
   CUDA_TRY(launch_sics(Q, K, p->sh, p->gp, p->st, t, p->num_sms, s));
   k_as_from_scratch<<<p->sh.BH, 32, 0, s>>>(p->sh, p->gp, scratch, as_out);
   CUDA_TRY(cudaGetLastError());
+  p->launches = 2;
   return SPADE_OK;
 }

@@ -261,7 +261,7 @@ k_gather(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, W
 // argmax (ties -> lowest candidate) unless forced, and the head's keep count / threshold.
 __global__ void __launch_bounds__(32)
 k_choose(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws,
-         const int* __restrict__ forced, int have_sics) {
+         const __grid_constant__ ForcedPack fp, int have_sics) {
   const int bh = blockIdx.x, lane = threadIdx.x;
   int best = 0;
   if (have_sics) {
@@ -285,7 +285,7 @@ k_choose(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
       if (sc > best_score) { best_score = sc; best = c; }
     }
   }
-  if (forced) best = forced[bh];
+  if (fp.on) best = (int)((fp.w[bh >> 3] >> ((bh & 7) * 4)) & 15u);
   if (lane == 0) {
     ws.scheme[bh] = best;
     const int nkb = gp.g[best].NBv;
@@ -949,17 +949,17 @@ cudaError_t launch_static(const Shape& sh, const GeoPack& gp, const StaticTables
   return cudaGetLastError();
 }
 
-cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, cudaStream_t s) {
+cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s) {
   const long total = (long)sh.BH * 2 * sh.NBmax * 32;
   long ctas = (total + 255) / 256;
-  if (ctas > 148 * 16) ctas = 148 * 16;
+  if (ctas > (long)num_sms * 16) ctas = (long)num_sms * 16;
   k_gather<<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
   return cudaGetLastError();
 }
 
 cudaError_t launch_choose(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
-                          const int* forced_dev, int have_sics, cudaStream_t s) {
-  k_choose<<<sh.BH, 32, 0, s>>>(sh, gp, st, ws, forced_dev, have_sics);
+                          const ForcedPack& forced, int have_sics, cudaStream_t s) {
+  k_choose<<<sh.BH, 32, 0, s>>>(sh, gp, st, ws, forced, have_sics);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   k_groups<<<1, 1024, 0, s>>>(sh, gp, ws, 0);
@@ -971,10 +971,10 @@ cudaError_t launch_groups_after_select(const Shape& sh, const GeoPack& gp, const
   return cudaGetLastError();
 }
 
-cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const WsTables& ws, cudaStream_t s) {
+cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s) {
   const long total = (long)sh.BH * 3 * sh.NBvmax;
   long ctas = (total + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
-  if (ctas > 148 * 8) ctas = 148 * 8;
+  if (ctas > (long)num_sms * 8) ctas = (long)num_sms * 8;
   k_pair_axis<<<(unsigned)ctas, WARPS_PER_CTA * 32, 0, s>>>(sh, gp, ws);
   return cudaGetLastError();
 }

@@ -88,6 +88,14 @@ struct WsTables {
 
 struct GeoPack { CandGeo g[SPADE_MAX_CANDS]; };
 
+// Forced schemes travel as a kernel argument (4 bits per head), so a launch -- also one captured in a
+// CUDA graph -- holds its own copy and no host array has to outlive the call.
+#define SPADE_MAX_BH 4096                        // B * heads a plan may have
+struct ForcedPack {
+  int on;                                        // 0: argmax of the Aggregation Score, 1: schemes packed below
+  uint32_t w[SPADE_MAX_BH / 8];
+};
+
 enum : uint32_t {
   SPADE_ST_OK = 0,
   SPADE_ST_TIMEOUT = 1,     // status[0]: a bounded wait gave up; status[1] = where, status[2] = item
@@ -100,10 +108,10 @@ cudaError_t launch_cells(const void* Q, const void* K, const Shape& sh, const Ws
 cudaError_t launch_blocks(const void* Q, const void* K, const Shape& sh, const GeoPack& gp, const StaticTables& st,
                           const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_static(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws, cudaStream_t s);
-cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, cudaStream_t s);
+cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_choose(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
-                          const int* forced_dev, int have_sics, cudaStream_t s);
-cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const WsTables& ws, cudaStream_t s);
+                          const ForcedPack& forced, int have_sics, cudaStream_t s);
+cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_groups_after_select(const Shape& sh, const GeoPack& gp, const WsTables& ws, cudaStream_t s);
 cudaError_t launch_summarize(const void* Q, const void* K, const Shape& sh, const GeoPack& gp, const StaticTables& st,
                              const WsTables& ws, int num_sms, cudaStream_t s);

@@ -8,6 +8,9 @@ Tolerances (also written where they are used):
   * index lists: exact as sets, except blocks whose block score is within 1e-4 (logit units,
     i.e. 1e-4 relative on the probability) of the cut; Top-P prefix lengths may differ only
     when the oracle's running mass at the cut is within 1e-4*p of p.  Excused blocks are counted.
+  * block scores of the mean estimator (Sec. 3.1, Fig. 4c), element by element: |S_gpu - S| <=
+    2e-6 * max_ij sum_c |Q'_ic K'_jc| / sqrt(d) (an fp32 sum of 128 products; a single TF32 product
+    of the summaries would be off by 2^-11 of that bound, 250 times the tolerance).
   * attention, given the GPU's own lists: max-abs 2e-2 and relative Frobenius 5e-3.
 """
 from __future__ import annotations
@@ -22,6 +25,7 @@ from oracle import spade_oracle as so
 from paper_2608_03335_b200 import binding
 from paper_2608_03335_b200.workloads import Workload, bf16_bits, make_qkv
 
+SCORE_REL = 2e-6          # of the largest sum of product magnitudes of the head
 ATTN_MAX_ABS = 2e-2
 ATTN_REL_FRO = 5e-3
 CUT_MARGIN = 1e-4
@@ -37,6 +41,7 @@ class Report:
     attn_max_abs: float = 0.0
     attn_rel_fro: float = 0.0
     sparsity: float = 0.0
+    score_err_rel: float = 0.0
 
 
 def make_plan(w: Workload, per_head=None, static=None, estimator="mean") -> binding.Plan:
@@ -160,6 +165,13 @@ def check_select(w: Workload, plan: binding.Plan, qb, kb, scheme, rep: Report, r
         g = so.geometry(w.grid, w.n_text, blk)
         sel = so.select_head(qb[bh], kb[bh], w.grid, w.n_text, blk, w.mode, value, static=static, estimator=estimator)
         nbv, nbt, nb = g["NBv"], g["NBt"], g["NB"]
+        if estimator == "mean":
+            # the estimator's table itself, element by element (Sec. 3.1, Fig. 4c)
+            S_gpu = t["block_scores"][bh, :nbv, :nbv].cpu().numpy()
+            bound = float((np.abs(sel["qs"][:nbv]) @ np.abs(sel["ks"][:nbv]).T).max()) / np.sqrt(w.d)
+            err = float(np.abs(S_gpu - sel["S"][:nbv, :nbv]).max())
+            assert err <= SCORE_REL * bound, f"head {bh}: block scores off by {err:.3e} (bound {SCORE_REL * bound:.3e})"
+            rep.score_err_rel = max(rep.score_err_rel, err / bound)
         # near-cut margin: 1e-4 on the mean estimator's O(1) scores; the max/min estimators add 128 products
         # of one sign pattern in fp32, so their rounding error grows with the score's magnitude
         margin = CUT_MARGIN if estimator == "mean" else max(CUT_MARGIN, 1e-5 * float(np.abs(sel["S"]).max()))

@@ -14,7 +14,7 @@ def _run(w, **kw):
     rep = run_layer_parity(w, **kw)
     print(f"[{w.name}] rows {rep.rows_checked} near-cut {rep.near_cut_blocks} scheme-ties {rep.scheme_ties} "
           f"attn blocks {rep.attn_blocks} max-abs {rep.attn_max_abs:.3e} rel-fro {rep.attn_rel_fro:.3e} "
-          f"sparsity {rep.sparsity:.4f}")
+          f"sparsity {rep.sparsity:.4f} score-err {rep.score_err_rel:.2e} of the magnitude bound")
     return rep
 
 
@@ -204,6 +204,36 @@ def test_full_size_paper_shapes_sampled():
     _run(WORKLOADS["paper_hunyuan"], rows_per_head=4, blocks_per_head=6, seed=16, attn_heads=[11])
 
 
+@pytest.mark.parametrize("cand", [0, 1, 2, 3])
+def test_full_size_sweep_forced_candidate_sparse(cand):
+    """Config 5 at its full shape (40 heads, N = 75 600): every head forced onto one candidate, target
+    sparsity 85 %.  Forced plans take the per-candidate summary pass instead of the cell tables; list
+    rows and query blocks are sampled, attention on three heads."""
+    from paper_2608_03335_b200.workloads import sweep_workload
+    w = sweep_workload(cand, 0.85)
+    rep = _run(w, forced=[cand] * w.heads, rows_per_head=6, blocks_per_head=8, seed=40 + cand, attn_heads=[0, 17, 39])
+    assert abs(rep.sparsity - 0.85) < 0.03
+
+
+@pytest.mark.parametrize("cand", [0, 1])
+def test_full_size_sweep_full_mask_is_dense_attention(cand):
+    """Config 5, target sparsity 0 on a 64-token and a 128-token candidate: every row lists every block
+    (row capacity = block count, 1440 K units per work item for 4x4x4), so the oracle fed the GPU's lists
+    evaluates Eq. 2 with M = 0, i.e. dense softmax attention (Eq. 1), on the sampled query blocks."""
+    from paper_2608_03335_b200.workloads import sweep_workload
+    w = sweep_workload(cand, 0.0)
+    rep = _run(w, forced=[cand] * w.heads, rows_per_head=4, blocks_per_head=8, seed=50 + cand, attn_heads=[3, 38])
+    assert abs(rep.sparsity) < 1e-12
+    assert rep.near_cut_blocks == 0
+
+
+def test_full_size_sweep_sparsest_point():
+    """Config 5 at 95 %: the shortest lists (72 of 1440 blocks for 4x4x4)."""
+    from paper_2608_03335_b200.workloads import sweep_workload
+    w = sweep_workload(0, 0.95)
+    _run(w, forced=[0] * w.heads, rows_per_head=6, blocks_per_head=8, seed=60, attn_heads=[11])
+
+
 @pytest.mark.parametrize("estimator", ["dsa", "dsa2"])
 def test_minmax_estimators_tiny_and_ragged(estimator):
     """Max / min summaries (bit-exact), the estimator's scores, the lists and the attention output."""
@@ -268,6 +298,42 @@ def test_layer_can_be_captured_in_a_cuda_graph_and_replayed():
             O.fill_(float("nan"))
             g.replay()
             torch.cuda.synchronize()
+            assert torch.equal(O, eager)
+        plan.spade_status()
+    finally:
+        plan.close()
+
+
+def test_captured_layer_with_forced_schemes_keeps_them_after_the_host_list_is_gone():
+    """Forced schemes travel inside the launch: a captured layer replays the schemes it was captured with,
+    whatever happens to the caller's (here pinned, then overwritten) host array afterwards."""
+    import ctypes as C
+    from paper_2608_03335_b200 import binding
+    from paper_2608_03335_b200.workloads import make_qkv
+    w = small_variant(WORKLOADS["wan14b"], heads=4, grid=(9, 10, 12))
+    Q, K, V = make_qkv(w, "cuda")
+    O = torch.empty_like(Q)
+    forced = [3, 0, 2, 1]
+    plan = binding.Plan(w.batch, w.heads, w.grid, w.n_text, w.candidates, w.mode, w.value)
+    try:
+        plan.spade_forward(Q, K, V, O, forced_scheme=forced)
+        torch.cuda.synchronize()
+        eager = O.clone()
+        host = torch.tensor(forced, dtype=torch.int32).pin_memory()           # truly asynchronous if it were copied
+        ptr = C.cast(host.data_ptr(), C.POINTER(C.c_int32))
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(s):
+            with torch.cuda.graph(g, stream=s):
+                binding._check(binding.lib().spade_forward(plan.handle, binding._ptr(Q), binding._ptr(K), binding._ptr(V),
+                                                            binding._ptr(O), plan._ws_ptr, binding._stream(s), ptr))
+        host.fill_(1)                                                          # the caller's list changes ...
+        for _ in range(2):
+            O.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            assert plan.tables()["scheme"].cpu().tolist() == forced           # ... the replay does not
             assert torch.equal(O, eager)
         plan.spade_status()
     finally:
