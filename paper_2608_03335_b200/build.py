@@ -8,7 +8,7 @@ import subprocess
 _PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_PKG, "csrc")
 LIB = os.path.join(_PKG, "libspade_b200.so")
-SOURCES = ["api.cu", "selection.cu", "scores.cu", "attn.cu"]
+SOURCES = ["api.cu", "plan.cu", "selection.cu", "scores.cu", "attn.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]

@@ -46,7 +46,7 @@ struct DeviceGuard {
   CUDA_TRY(guard__.err)
 
 struct WsLayout {
-  size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, scores, colkeep, rowfull, pair_axis, pair_union, mm, text_start, head_work, att_scratch;
+  size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, nsum, scores, colkeep, rowfull, pair_axis, pair_union, mm, text_start, head_work, att_scratch;
   size_t bytes;
 };
 
@@ -61,6 +61,11 @@ struct spade_plan_s {
   StaticTables st;
   void* d_static;        // one allocation holding rowoff, nvalid, kvalid, budget
   WsLayout lay;
+  PlanFusedCfg pf;       // one-pass scheme generation (plan.cu), when the candidate set fits it
+  PlanMaps* pmaps;       // its tensor maps for the last (Q, K) seen
+  void* d_pf;            // its output tables (device): int rows, then float reciprocals of the block sizes
+  size_t pf_entries;
+  const void *pq, *pk;
   ScoreMaps* smaps;      // tensor map of the K' summaries inside `smaps_ws`
   const void* smaps_ws;
   AttnMaps* maps;        // host copy of the TMA descriptors for the last (Q,K,V,O) seen
@@ -101,6 +106,7 @@ WsTables tables_at(const spade_plan_s* p, void* ws) {
   t.text_start = (int*)(b + l.text_start);
   t.cells = (float*)(b + l.cells);
   t.csum = (float*)(b + l.csum);
+  t.nsum = (float*)(b + l.nsum);
   t.scores = (float*)(b + l.scores);
   t.pair_axis = (int*)(b + l.pair_axis);
   t.pair_union = (int*)(b + l.pair_union);
@@ -151,8 +157,9 @@ void compute_layout(spade_plan_s* p) {
   l.qsum = take((size_t)BH * sh.NBmax * SPADE_D * 4);
   l.ksum = take((size_t)BH * sh.NBmax * SPADE_D * 4);
   l.kv_idx = take((size_t)BH * sh.NBmax * sh.cap * 4);
-  l.cells = take(sh.use_cells ? (size_t)BH * 2 * sh.NCELL * 2 * SPADE_D * 4 : 0);
-  l.csum = take(sh.use_cells ? (size_t)BH * 2 * n_cands * sh.NBmax * SPADE_D * 4 : 0);
+  l.cells = take(sh.use_cells && !p->pf.on ? (size_t)BH * 2 * sh.NCELL * 2 * SPADE_D * 4 : 0);
+  l.csum = take(sh.use_cells || p->pf.on ? (size_t)BH * 2 * n_cands * sh.NBmax * SPADE_D * 4 : 0);
+  l.nsum = take(p->pf.on ? (size_t)BH * 2 * n_cands * sh.NBmax * SPADE_D * 4 : 0);
   sh.ld_scores = (sh.NBvmax + 63) & ~63;
   l.scores = take((size_t)BH * sh.NBvmax * sh.ld_scores * 4);
   l.mm = take(sh.estimator ? (size_t)4 * BH * SPADE_D * sh.ld_scores * 4 : 0);
@@ -330,12 +337,24 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
   p->st.budget = (const float*)(base + o_budget);
 
   p->base_cap = sh.cap;
+  plan_fused_configure(&p->pf, sh, p->gp, p->num_sms);
+  if (p->pf.on) {
+    std::vector<int> pe;
+    std::vector<float> pi;
+    plan_fused_tables(p->pf, sh, p->gp, pe, pi);
+    p->pf_entries = pe.size();
+    e = cudaMalloc(&p->d_pf, pe.size() * 8);
+    if (e == cudaSuccess) e = cudaMemcpy(p->d_pf, pe.data(), pe.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy((char*)p->d_pf + pe.size() * 4, pi.data(), pi.size() * 4, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { cudaFree(p->d_pf); cudaFree(p->d_static); free(p); return fail(SPADE_ERR_CUDA, "table upload: %s", cudaGetErrorString(e)); }
+  }
   compute_layout(p);
 
   p->maps = (AttnMaps*)calloc(1, attn_maps_bytes());
   p->smaps = (ScoreMaps*)calloc(1, score_maps_bytes());
-  if (!p->maps || !p->smaps) {
-    cudaFree(p->d_static); free(p->maps); free(p->smaps); free(p);
+  p->pmaps = (PlanMaps*)calloc(1, plan_maps_bytes());
+  if (!p->maps || !p->smaps || !p->pmaps) {
+    cudaFree(p->d_static); free(p->maps); free(p->smaps); free(p->pmaps); free(p);
     return fail(SPADE_ERR_INVALID_ARG, "out of host memory");
   }
   *out = p;
@@ -345,6 +364,7 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
 int spade_plan_destroy(spade_plan_t* p) {
   if (!p) return SPADE_OK;
   cudaFree(p->d_static);
+  cudaFree(p->d_pf);
   if (p->host_ready) {
     cudaStreamDestroy(p->copy_in);
     cudaStreamDestroy(p->copy_out);
@@ -353,6 +373,7 @@ int spade_plan_destroy(spade_plan_t* p) {
   }
   free(p->maps);
   free(p->smaps);
+  free(p->pmaps);
   free(p);
   return SPADE_OK;
 }
@@ -435,7 +456,17 @@ int spade_plan(spade_plan_t* p, const void* Q, const void* K, void* ws, void* st
   }
   p->have_csum = 0;
   if (!skip_sics) {
-    if (p->sh.use_cells) {
+    if (p->pf.on) {
+      if (Q != p->pq || K != p->pk) {
+        char msg[256];
+        if (plan_encode_maps(p->pmaps, Q, K, p->sh, p->pf, msg, sizeof(msg))) return fail(SPADE_ERR_CUDA, "tensor map: %s", msg);
+        p->pq = Q; p->pk = K;
+      }
+      CUDA_TRY(launch_plan_fused(p->pmaps, Q, K, p->sh, p->gp, p->st, t, p->pf, p->num_sms, (const int*)p->d_pf,
+                                 (const float*)((const char*)p->d_pf + p->pf_entries * 4), s));
+      p->launches += 2;
+      p->have_csum = 1;
+    } else if (p->sh.use_cells) {
       CUDA_TRY(launch_cells(Q, K, p->sh, t, p->num_sms, s));
       CUDA_TRY(launch_blocks(Q, K, p->sh, p->gp, p->st, t, p->num_sms, s));
       p->launches += 2;
@@ -583,6 +614,7 @@ int spade_forward_host(spade_plan_t* p, const void* hQ, const void* hK, const vo
     view.keep_status = g > 0;
     view.stage = 0; view.stage_ws = nullptr; view.smaps_ws = nullptr;
     view.mq = view.mk = view.mv = view.mo = nullptr;
+    view.pq = view.pk = nullptr;
     compute_layout(&view);
     CUDA_TRY(cudaStreamWaitEvent(s, p->ev_in[g], 0));
     rc = spade_forward(&view, (char*)dQ + off, (char*)dK + off, (char*)dV + off, (char*)dO + off, ws, stream,
@@ -595,6 +627,7 @@ int spade_forward_host(spade_plan_t* p, const void* hQ, const void* hK, const vo
   }
   // the views overwrote the shared descriptors and laid the workspace out for fewer heads
   p->mq = p->mk = p->mv = p->mo = nullptr;
+  p->pq = p->pk = nullptr;
   p->smaps_ws = nullptr;
   p->stage = 0; p->stage_ws = nullptr;
   p->launches = launches;

@@ -59,6 +59,35 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   }
 }
 
+// The same bounded wait for barriers that are expected to take microseconds (a copy from HBM): sleeps a
+// little between polls so that waiting warps leave the issue slots to the working ones.
+__device__ __forceinline__ bool mbar_wait_sleepy(uint64_t* bar, uint32_t parity, volatile uint32_t* abort, uint64_t limit_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  uint32_t spins = 0;
+  long long t0 = 0;
+  for (;;) {
+    __nanosleep(40);
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 63u) == 0) {
+      if (*abort) return false;
+      const long long now = clock64();
+      if (t0 == 0) t0 = now;
+      else if ((uint64_t)(now - t0) > 2ull * limit_ns) { *abort = 1; return false; }
+    }
+  }
+}
+
+// A whole warp waits, one lane polls: lane 0 runs the bounded wait (sleeping between polls), the others park
+// at the warp barrier instead of hammering the barrier unit; afterwards every lane observes the completed
+// phase itself (one poll that succeeds), which orders its later reads after the barrier.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort, uint64_t limit_ns) {
+  uint32_t ok = 1;
+  if ((threadIdx.x & 31) == 0) ok = mbar_wait_sleepy(bar, parity, abort, limit_ns) ? 1u : 0u;
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  if (ok) ok = mbar_try_wait(bar, parity) ? 1u : 0u;
+  return __all_sync(0xffffffffu, ok != 0);
+}
+
 // ---- proxies / fences --------------------------------------------------------------------------
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #define SPADE_MAX_CANDS 8
 #define SPADE_MAX_NB 2048          // blocks per head (video + text) the kernels are sized for
 #define SPADE_D 128
@@ -77,6 +79,7 @@ struct WsTables {
   int* text_start;      // [BH+1] prefix of the text query tiles over head_order (they are scheduled first)
   float* cells;         // [BH][2 tensors][NCELL][2 (sum of q/|q|, sum of q)][128]
   float* csum;          // [BH][2 tensors][C][NBmax][128] mean summaries of every candidate
+  float* nsum;          // same shape: sum over a block's tokens of q / |q| (one-pass scheme generation only)
   int* pair_axis;       // [BH] axis (0 t, 1 h, 2 w) along which 64-token query blocks are paired into 128-row tiles
   int* pair_union;      // [BH][3] total merged-list length for each pairing axis
   uint8_t* colkeep;     // [BH][NBmax] KV block kept by every query block (intra rule on K, sink)
@@ -101,6 +104,29 @@ enum : uint32_t {
   SPADE_ST_TIMEOUT = 1,     // status[0]: a bounded wait gave up; status[1] = where, status[2] = item
 };
 
+// Configuration of the one-pass scheme-generation kernel (plan.cu); on = 0 when the candidate set does not
+// fit it (a block footprint above 128 tokens in the (h, w) plane, more than 64 blocks of all candidates in one
+// column slice) and the cell tables serve instead.
+struct PlanFusedCand {
+  int lbt, bt_mask;        // log2(bt), bt - 1
+  int lbh, lbw;            // log2 of the block extents along h and w
+  int cbw, lcbw, nblk;     // blocks per column along w (and its log2), blocks per column slice
+  int slot_base;           // first slot of this candidate's blocks among the slots of a slice
+};
+struct PlanFusedCfg {
+  int on;
+  int colH, colW, lcolW;   // column footprint in the (h, w) plane: 128 tokens, a multiple of every candidate's (bh, bw)
+  int ncol_h, ncol_w;      // columns over the grid
+  int tchunk, nchunks;     // slices per work item (a multiple of every candidate's bt) and chunks over T
+  int stages;              // ring of slices in shared memory
+  int nblk;                // slots: blocks of all candidates in one column slice
+  int cpw;                 // 32-column chunks (8 slots each) per epilogue warpgroup; rows of the weight matrix = 64 * cpw
+  int nrows;
+  int text_blocks;         // text blocks over all candidates
+  PlanFusedCand cand[SPADE_MAX_CANDS];
+  unsigned char slot_cand[64];   // slot -> candidate
+};
+
 // ---- launchers (definitions in the .cu files) ------------------------------------------------
 cudaError_t launch_sics(const void* Q, const void* K, const Shape& sh, const GeoPack& gp, const StaticTables& st,
                         const WsTables& ws, int num_sms, cudaStream_t s);
@@ -120,6 +146,17 @@ cudaError_t launch_minmax(const void* Q, const void* K, const Shape& sh, const G
 cudaError_t launch_scores_minmax(const Shape& sh, const GeoPack& gp, const WsTables& ws, cudaStream_t s);
 cudaError_t launch_select(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
                           cudaStream_t s);
+
+struct PlanMaps;   // tensor maps of Q and K for the one-pass scheme generation, defined in plan.cu
+size_t plan_maps_bytes();
+void plan_fused_configure(PlanFusedCfg* cfg, const Shape& sh, const GeoPack& gp, int num_sms);
+int plan_encode_maps(PlanMaps* out, const void* Q, const void* K, const Shape& sh, const PlanFusedCfg& cfg, char* err,
+                     size_t errlen);
+void plan_fused_tables(const PlanFusedCfg& cfg, const Shape& sh, const GeoPack& gp, std::vector<int>& e,
+                       std::vector<float>& inv);
+cudaError_t launch_plan_fused(const PlanMaps* maps, const void* Q, const void* K, const Shape& sh, const GeoPack& gp,
+                              const StaticTables& st, const WsTables& ws, const PlanFusedCfg& cfg, int num_sms,
+                              const int* tab_e, const float* tab_inv, cudaStream_t s);
 
 struct ScoreMaps;  // tensor map of the K' summaries, defined in scores.cu
 size_t score_maps_bytes();

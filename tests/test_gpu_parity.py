@@ -14,7 +14,7 @@ def _run(w, **kw):
     rep = run_layer_parity(w, **kw)
     print(f"[{w.name}] rows {rep.rows_checked} near-cut {rep.near_cut_blocks} scheme-ties {rep.scheme_ties} "
           f"attn blocks {rep.attn_blocks} max-abs {rep.attn_max_abs:.3e} rel-fro {rep.attn_rel_fro:.3e} "
-          f"sparsity {rep.sparsity:.4f} score-err {rep.score_err_rel:.2e} of the magnitude bound")
+          f"sparsity {rep.sparsity:.4f} score-err {rep.score_err_rel:.2e} (kernel alone {rep.score_err_kernel:.2e}) of the magnitude bound")
     return rep
 
 
