@@ -184,6 +184,14 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
     // ================= token warps: |q_t|^2 and the three pieces of 1/|q_t| into the weight matrix ========
     const int tok = tid;
     const int dh = tok >> cfg.lcolW, dw = tok & (cfg.colW - 1);
+    uint32_t woff[4][3];                       // where this token's three pieces go, per candidate
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const PlanFusedCand& pc = cfg.cand[c < sh.C ? c : 0];
+      const int slot = pc.slot_base + ((dh >> pc.lbh) << pc.lcbw) + (dw >> pc.lbw);
+#pragma unroll
+      for (int pce = 0; pce < 3; ++pce) woff[c][pce] = pf_w_offset(NROWS, pf_row(CPW, slot, pce), tok);
+    }
     uint32_t i = 0;
     for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
       const int chunk = (item / col_items) % cfg.nchunks;
@@ -226,7 +234,14 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
         const uint16_t r3 = pf_bf16(e1 - pf_bf16_to_float(r2));
         if (!ptx::mbar_wait_warp(&ctl.w_empty[b], ph ^ 1, &ctl.abort, PF_WAIT_NS)) { site = 206; break; }
         uint8_t* wb = wmat + b * W_BYTES;
-        for (int c = 0; c < sh.C; ++c) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {                                    // the first four candidates: offsets kept in registers
+          if (c >= sh.C) break;
+          *reinterpret_cast<uint16_t*>(wb + woff[c][0]) = r1;
+          *reinterpret_cast<uint16_t*>(wb + woff[c][1]) = r2;
+          *reinterpret_cast<uint16_t*>(wb + woff[c][2]) = r3;
+        }
+        for (int c = 4; c < sh.C; ++c) {
           const PlanFusedCand& pc = cfg.cand[c];
           const int slot = pc.slot_base + ((dh >> pc.lbh) << pc.lcbw) + (dw >> pc.lbw);
           const int n0 = pf_row(CPW, slot, 0);
