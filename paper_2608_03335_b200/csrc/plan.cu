@@ -373,18 +373,28 @@ k_sics_from_sums(const __grid_constant__ Shape sh, const __grid_constant__ GeoPa
   const int lane = threadIdx.x & 31;
   const long gw = (long)blockIdx.x * 8 + (threadIdx.x >> 5), nw = (long)gridDim.x * 8;
   const long total = (long)sh.BH * 2 * sh.units_per_ht;
-  for (long u = gw; u < total; u += nw) {
-    const int ht = (int)(u / sh.units_per_ht), rem = (int)(u % sh.units_per_ht);
-    int c = 0;
+  for (long u0 = gw * 4; u0 < total; u0 += nw * 4) {           // four blocks per warp and step: four loads in flight
+    float4 v[4];
+    size_t out[4];
 #pragma unroll
-    for (int i = 1; i < SPADE_MAX_CANDS; ++i)
-      if (i < sh.C && rem >= gp.g[i].unit_off) c = i;
-    const int b = rem - gp.g[c].unit_off;
-    const float4 v = __ldcs(reinterpret_cast<const float4*>(ws.nsum + ((((size_t)ht * sh.C + c) * sh.NBmax) + b) * SPADE_D) + lane);
-    float s = (v.x * v.x + v.y * v.y) + (v.z * v.z + v.w * v.w);
+    for (int q = 0; q < 4; ++q) {
+      const long u = u0 + q < total ? u0 + q : total - 1;
+      const int ht = (int)(u / sh.units_per_ht), rem = (int)(u % sh.units_per_ht);
+      int c = 0;
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(FULL, s, o);
-    if (lane == 0) ws.sics[(((size_t)(ht >> 1) * sh.C + c) * 2 + (ht & 1)) * sh.NBvmax + b] = s;
+      for (int i = 1; i < SPADE_MAX_CANDS; ++i)
+        if (i < sh.C && rem >= gp.g[i].unit_off) c = i;
+      const int b = rem - gp.g[c].unit_off;
+      v[q] = __ldcs(reinterpret_cast<const float4*>(ws.nsum + ((((size_t)ht * sh.C + c) * sh.NBmax) + b) * SPADE_D) + lane);
+      out[q] = (((size_t)(ht >> 1) * sh.C + c) * 2 + (ht & 1)) * sh.NBvmax + b;
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float s = (v[q].x * v[q].x + v[q].y * v[q].y) + (v[q].z * v[q].z + v[q].w * v[q].w);
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(FULL, s, o);
+      if (lane == 0 && u0 + q < total) ws.sics[out[q]] = s;
+    }
   }
 }
 
@@ -522,7 +532,7 @@ cudaError_t launch_plan_fused(const PlanMaps* maps, const void* Q, const void* K
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const long blocks = (long)sh.BH * 2 * sh.units_per_ht;
-  long ctas = (blocks + 7) / 8;
+  long ctas = (blocks + 31) / 32;
   if (ctas > (long)num_sms * 8) ctas = (long)num_sms * 8;
   k_sics_from_sums<<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
   return cudaGetLastError();

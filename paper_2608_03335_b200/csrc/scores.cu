@@ -3,8 +3,8 @@
 //
 // The summaries are fp32 and the selection must agree with an fp64 evaluation to 1e-4 in the logits,
 // so a plain TF32 product (10-bit mantissa) is not enough.  Each operand is split x = hi + lo with
-// hi = x truncated to TF32 and lo = x - hi (exact in fp32); the product uses the three terms
-// hi*hi + hi*lo + lo*hi (the dropped lo*lo term is 2^-22 relative), all accumulated in one fp32
+// hi = x rounded to the nearest TF32 value and lo = x - hi (exact in fp32); the product uses the three terms
+// hi*hi + hi*lo + lo*hi (the dropped lo*lo term is at most 2^-22 relative, of either sign), all accumulated in one fp32
 // TMEM tile by tcgen05.mma kind::tf32.  A (128 query blocks x 128 channels, hi and lo) lives in TMEM,
 // B (64 KV blocks x 128 channels) arrives by TMA in two stages and is split in place in shared memory.
 // Warp 4 issues the TMA loads and the products; warps 0-3 stage A, split B and write the scores, so the
@@ -24,6 +24,7 @@ constexpr int SC_N = 64;                         // KV blocks per column tile
 constexpr int SC_SUB = SC_N * 128;               // bytes of one 32-channel sub-tile (64 rows x 128 B)
 constexpr int SC_STAGE = 8 * SC_SUB;             // hi (4 sub-tiles) + lo (4 sub-tiles) = 64 KB
 constexpr uint64_t SC_WAIT_NS = 2000000000ull;
+constexpr int SC_PARTS = 3;                      // work items per row tile (balance over the SMs)
 constexpr int SC_NST = 3;                        // shared-memory stages of B (D stays double-buffered in TMEM)
 constexpr size_t SC_SMEM = SC_NST * SC_STAGE + 1024 + 256;
 
@@ -74,16 +75,19 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
   ptx::tc_fence_after();
   const uint32_t tm = ctl.tmem_base;                 // A hi: cols 0..127, A lo: 128..255, D: 256..319 and 320..383
   const int row_tiles = (sh.NBvmax + 127) / 128;
-  const int items = sh.BH * row_tiles;
+  const int items = sh.BH * row_tiles * SC_PARTS;     // a row tile's column tiles are split over SC_PARTS work items
   uint32_t tiles_done = 0;                            // column tiles so far (same in every role)
   uint32_t items_done = 0;
   uint32_t site = 0;
 
   for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
-    const int bh = item / row_tiles, rt = item % row_tiles;
+    const int part = item % SC_PARTS, rt = (item / SC_PARTS) % row_tiles, bh = item / (SC_PARTS * row_tiles);
     const int nbv = gp.g[ws.scheme[bh]].NBv;
     if (rt * 128 >= nbv) continue;
-    const int n_ct = (nbv + SC_N - 1) / SC_N;
+    const int n_ct_all = (nbv + SC_N - 1) / SC_N, per_part = (n_ct_all + SC_PARTS - 1) / SC_PARTS;
+    const int ct0 = part * per_part;
+    const int n_ct = min(per_part, n_ct_all - ct0);
+    if (n_ct <= 0) continue;
     if (warp == 4) {
       // ================= issuer: K' tiles by TMA, products, commits ===================================
       if (lane == 0) {
@@ -92,7 +96,7 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
         auto load_tile = [&](int ct) {                 // the stage of tile ct must be free
           const uint32_t st = (tiles_done + ct) % SC_NST;
           ptx::mbar_expect_tx(&ctl.b_full[st], 4 * SC_SUB);
-          for (int s = 0; s < 4; ++s) ptx::tma_load_3d(smem + st * SC_STAGE + s * SC_SUB, &maps.k, &ctl.b_full[st], 32 * s, ct * SC_N, bh);
+          for (int s = 0; s < 4; ++s) ptx::tma_load_3d(smem + st * SC_STAGE + s * SC_SUB, &maps.k, &ctl.b_full[st], 32 * s, (ct0 + ct) * SC_N, bh);
         };
         // every stage is free here: all products of the previous item were waited for below
         for (int ct = 0; ct < SC_NST && ct < n_ct; ++ct) load_tile(ct);
@@ -142,7 +146,7 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
             const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const uint32_t h = __float_as_uint(x[e]) & 0xffffe000u;
+              const uint32_t h = (__float_as_uint(x[e]) + 0x1000u) & 0xffffe000u;      // nearest TF32 value
               hi[q * 4 + e] = h;
               lo[q * 4 + e] = __float_as_uint(x[e] - __uint_as_float(h));
             }
@@ -164,10 +168,10 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
           uint4* bl_ = reinterpret_cast<uint4*>(smem + st * SC_STAGE + 4 * SC_SUB);
           for (int i = tid; i < 4 * SC_SUB / 16; i += 128) {
             uint4 v = bh_[i], h, l;
-            h.x = v.x & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
-            h.y = v.y & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
-            h.z = v.z & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
-            h.w = v.w & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
+            h.x = (v.x + 0x1000u) & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
+            h.y = (v.y + 0x1000u) & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
+            h.z = (v.z + 0x1000u) & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
+            h.w = (v.w + 0x1000u) & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
             bh_[i] = h;
             bl_[i] = l;
           }
@@ -180,7 +184,7 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
           const uint32_t tp = t - 1, sp = tp & 1;
           if (!__all_sync(0xffffffffu, ptx::mbar_wait(&ctl.mma_done[sp], (tp >> 1) & 1, &ctl.abort, SC_WAIT_NS))) { site = 106; break; }
           ptx::tc_fence_after();
-          float* dst = ws.scores + ((size_t)bh * sh.NBvmax + row) * sh.ld_scores + (ct - 1) * SC_N;
+          float* dst = ws.scores + ((size_t)bh * sh.NBvmax + row) * sh.ld_scores + (ct0 + ct - 1) * SC_N;
 #pragma unroll
           for (int ch = 0; ch < 2; ++ch) {
             uint32_t r[32];
@@ -247,7 +251,7 @@ cudaError_t launch_scores(const ScoreMaps* maps, const Shape& sh, const GeoPack&
                           cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(k_scores, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
   if (e != cudaSuccess) return e;
-  const int items = sh.BH * ((sh.NBvmax + 127) / 128);
+  const int items = sh.BH * ((sh.NBvmax + 127) / 128) * SC_PARTS;
   const int grid = items < num_sms ? items : num_sms;
   k_scores<<<grid, SC_THREADS, SC_SMEM, s>>>(*maps, sh, gp, ws, 1.0f / sqrtf((float)SPADE_D));
   return cudaGetLastError();

@@ -257,29 +257,36 @@ k_gather(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, W
   }
 }
 
-// One warp per head: AS(X|c) = sum_b SICS (Eq. 3; fixed lane-strided order), normalised score,
-// argmax (ties -> lowest candidate) unless forced, and the head's keep count / threshold.
-__global__ void __launch_bounds__(32)
+// One CTA per head: AS(X|c) = sum_b SICS (Eq. 3; fixed lane-strided order, one warp per (candidate, tensor)),
+// then warp 0: normalised score, argmax (ties -> lowest candidate) unless forced, and the head's keep count /
+// threshold.
+__global__ void __launch_bounds__(256)
 k_choose(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws,
          const __grid_constant__ ForcedPack fp, int have_sics) {
-  const int bh = blockIdx.x, lane = threadIdx.x;
+  __shared__ float as_sm[SPADE_MAX_CANDS * 2];
+  const int bh = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (have_sics) {
+    for (int ct = warp; ct < sh.C * 2; ct += 8) {
+      const int c = ct >> 1, t = ct & 1;
+      const float* p = ws.sics + (((size_t)bh * sh.C + c) * 2 + t) * sh.NBvmax;
+      float s = 0.f;
+      for (int b = lane; b < gp.g[c].NBv; b += 32) s += p[b];
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(FULL, s, o);
+      if (lane == 0) as_sm[ct] = s;
+    }
+  }
+  __syncthreads();
+  if (warp != 0) return;
   int best = 0;
   if (have_sics) {
     float best_score = -1e30f;
     for (int c = 0; c < sh.C; ++c) {
-      float a[2];
-      for (int t = 0; t < 2; ++t) {
-        const float* p = ws.sics + (((size_t)bh * sh.C + c) * 2 + t) * sh.NBvmax;
-        float s = 0.f;
-        for (int b = lane; b < gp.g[c].NBv; b += 32) s += p[b];
-#pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(FULL, s, o);
-        a[t] = s;
-      }
-      const float sc = (a[0] + a[1]) * gp.g[c].inv_z;
+      const float a0 = as_sm[2 * c], a1 = as_sm[2 * c + 1];
+      const float sc = (a0 + a1) * gp.g[c].inv_z;
       if (lane == 0) {
-        ws.as[((size_t)bh * sh.C + c) * 2 + 0] = a[0];
-        ws.as[((size_t)bh * sh.C + c) * 2 + 1] = a[1];
+        ws.as[((size_t)bh * sh.C + c) * 2 + 0] = a0;
+        ws.as[((size_t)bh * sh.C + c) * 2 + 1] = a1;
         ws.score[(size_t)bh * sh.C + c] = sc;
       }
       if (sc > best_score) { best_score = sc; best = c; }
@@ -674,6 +681,8 @@ k_scores_minmax(const __grid_constant__ Shape sh, const __grid_constant__ GeoPac
 // ------------------------------------------------------------------------------------------------
 // Estimator + index search.
 constexpr int SEL_R = 8;        // query-block rows per CTA; one warp per row
+constexpr int SEL_CAND = 256;   // keys of the bin the cut falls in that the later radix passes work on
+constexpr int SEL_WARP_WORDS = 256 + 512 + SEL_CAND;   // per warp: bin counts, 64-bit bin masses, candidate keys
 
 __device__ __forceinline__ uint32_t order_key(float s) {      // larger float <=> larger key
   const uint32_t u = __float_as_uint(s);
@@ -772,8 +781,9 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
     return;
   }
   const float* s = sc + warp * ldc;
-  int* hcnt = reinterpret_cast<int*>(sk) + warp * 512;
-  float* hmass = reinterpret_cast<float*>(hcnt + 256);
+  int* hcnt = reinterpret_cast<int*>(sk) + warp * (sh.mode == 1 ? SEL_WARP_WORDS : SEL_WARP_WORDS - 512);   // [256] counts per radix bin
+  unsigned long long* hmass = reinterpret_cast<unsigned long long*>(hcnt + 256);     // [256] softmax mass per bin, fixed point
+  uint32_t* cand = reinterpret_cast<uint32_t*>(hcnt + (sh.mode == 1 ? 768 : 256));   // [SEL_CAND] rel keys still in the race (over the unused masses in Top-K mode)
   const unsigned lt = (1u << lane) - 1u;
 
   // Keys replace the scores in place; the radix descent starts below the bits every key of the row
@@ -792,10 +802,29 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
     kmin = min(kmin, __shfl_xor_sync(FULL, kmin, o));
   }
   __syncwarp();
-  int hi = (kmax ^ kmin) ? 32 - __clz(kmax ^ kmin) : 0;        // bits [hi, 32) are common to the row
-  uint32_t T = hi < 32 ? ((kmax >> hi) << hi) : 0u;             // becomes the key of the last kept value
+  // The descent works on rel = key - kmin, whose top bits spread over the row's actual range of values
+  // (a common bit prefix would not: rows that straddle zero differ in the sign bit already).
+  int hi = kmax != kmin ? 32 - __clz(kmax - kmin) : 0;         // rel < 2^hi
+  uint32_t T = 0u;                                              // becomes rel of the last kept value
   int need = 0;         // how many blocks with key == T are kept (lowest ids first)
   bool all = false;
+  // The first pass of the descent scans the whole row.  As soon as the bin the cut falls in holds at most
+  // SEL_CAND keys they are copied out, and the remaining passes (down to bit 0) only touch that short list.
+  int m = -1;           // -1: the candidates are the whole row; >= 0: cand[0 .. m)
+  auto compact = [&](int cnt) {
+    if (m >= 0 || hi == 0 || cnt > SEL_CAND) return;
+    int at = 0;
+    for (int j0 = 0; j0 < n; j0 += 32) {
+      const int j = j0 + lane;
+      const uint32_t key = j < n ? ks[j] - kmin : 0u;
+      const bool hit = j < n && (key >> hi) == (T >> hi);
+      const unsigned bm = __ballot_sync(FULL, hit);
+      if (hit) cand[at + __popc(bm & lt)] = key;
+      at += __popc(bm);
+    }
+    m = at;
+    __syncwarp();
+  };
   if (sh.mode != 1) {
     // Top-K: radix select of the k-th largest key, up to 8 bits per pass.
     need = ws.keep[bh];
@@ -805,8 +834,11 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
       const uint32_t bmask = (1u << (hi - lo)) - 1u;
       for (int i = lane; i < 256; i += 32) hcnt[i] = 0;
       __syncwarp();
-      for (int j = lane; j < n; j += 32) {
-        const uint32_t key = ks[j];
+      const int cnt_all = m < 0 ? n : m;
+      const uint32_t* src = m < 0 ? ks : cand;
+      const uint32_t base = m < 0 ? kmin : 0u;                     // the candidate list holds rel already
+      for (int j = lane; j < cnt_all; j += 32) {
+        const uint32_t key = src[j] - base;
         if (hi >= 32 || (key >> hi) == (T >> hi)) atomicAdd(&hcnt[(key >> lo) & bmask], 1);
       }
       __syncwarp();
@@ -816,60 +848,57 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
       T |= (uint32_t)bin << lo;
       need -= above;
       hi = lo;
+      const int cnt = hcnt[bin];
       __syncwarp();
+      compact(cnt);
     }
   } else {
-    // Top-P: same descent, on softmax mass.  Weights exp(s - max); target = p * sum.
-    const float m = key_to_float(kmax);
-    float z = 0.f;
-    for (int j = lane; j < n; j += 32) z += expf(key_to_float(ks[j]) - m);
+    // Top-P: the same descent on softmax mass.  Weights exp(s - max) are summed in 2^-40 fixed point:
+    // integer sums do not depend on the order the lanes add them in, so the lists are reproducible bit for
+    // bit, and the mass of a bin equals the sum of its sub-bins in the next pass exactly.
+    const float mx = key_to_float(kmax);
+    auto weight = [&](uint32_t rel) -> unsigned long long {
+      return __float2ull_rn(expf(key_to_float(rel + kmin) - mx) * 1099511627776.f);
+    };
+    unsigned long long z = 0ull;
+    for (int j = lane; j < n; j += 32) z += weight(ks[j] - kmin);
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) z += __shfl_xor_sync(FULL, z, o);
-    const float target = ws.pthr[bh] * z;
-    float above = 0.f;
+    unsigned long long target = (unsigned long long)ceil((double)ws.pthr[bh] * (double)z);
+    if (target > z) target = z;
+    if (target == 0ull) target = 1ull;
+    unsigned long long above = 0ull;
     int cnt_T = n;
-    bool first = true;
-    if (hi == 0 && z < target) all = true;               // identical scores and p above the total
     while (hi > 0 && !all) {
       const int lo = hi > 8 ? hi - 8 : 0;
       const uint32_t bmask = (1u << (hi - lo)) - 1u;
-      for (int i = lane; i < 256; i += 32) { hcnt[i] = 0; hmass[i] = 0.f; }
+      for (int i = lane; i < 256; i += 32) { hcnt[i] = 0; hmass[i] = 0ull; }
       __syncwarp();
-      for (int j = lane; j < n; j += 32) {
-        const uint32_t key = ks[j];
+      const int cnt_all = m < 0 ? n : m;
+      const uint32_t* src = m < 0 ? ks : cand;
+      const uint32_t base = m < 0 ? kmin : 0u;
+      for (int j = lane; j < cnt_all; j += 32) {
+        const uint32_t key = src[j] - base;
         if (hi >= 32 || (key >> hi) == (T >> hi)) {
           atomicAdd(&hcnt[(key >> lo) & bmask], 1);
-          atomicAdd(&hmass[(key >> lo) & bmask], expf(key_to_float(key) - m));
+          atomicAdd(&hmass[(key >> lo) & bmask], weight(key));
         }
       }
       __syncwarp();
-      int bin = find_bin<float>(hmass, target, above, lane);
-      if (bin < 0) {
-        if (first) { all = true; break; }              // the total never reaches p: keep everything
-        // rounding between passes: the crossing bin of the previous pass is consumed whole, so the
-        // cut falls in its lowest non-empty sub-bin; everything above that sub-bin counts as kept.
-        int lowest = 256;
-        float tot = 0.f;
-        for (int i = lane; i < 256; i += 32) { if (hcnt[i] > 0) lowest = min(lowest, i); tot += hmass[i]; }
-#pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) {
-          lowest = min(lowest, __shfl_xor_sync(FULL, lowest, o));
-          tot += __shfl_xor_sync(FULL, tot, o);
-        }
-        if (lowest > 255) { all = true; break; }       // no key under the prefix (cannot happen): keep the row whole
-        bin = lowest;
-        above += tot - hmass[bin];
-      }
+      const int bin = find_bin<unsigned long long>(hmass, target, above, lane);
+      if (bin < 0) { all = true; break; }            // cannot happen (target <= total mass under the prefix)
       T |= (uint32_t)bin << lo;
       cnt_T = hcnt[bin];
       hi = lo;
-      first = false;
       __syncwarp();
+      compact(cnt_T);
     }
     if (!all) {
-      const float wT = expf(key_to_float(T) - m);
-      float t = wT > 0.f ? ceilf((target - above) / wT) : (float)cnt_T;
-      need = (int)fminf(fmaxf(t, 1.f), (float)cnt_T);
+      // every key equal to T carries the same weight: how many of them (lowest ids first) the mass still needs
+      const unsigned long long wT = weight(T);
+      unsigned long long t = wT > 0ull ? (target - above + wT - 1ull) / wT : (unsigned long long)cnt_T;
+      if (target <= above) t = 1ull;
+      need = (int)(t < 1ull ? 1ull : (t > (unsigned long long)cnt_T ? (unsigned long long)cnt_T : t));
     }
   }
 
@@ -885,7 +914,7 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
     for (int j0 = 0; j0 < n; j0 += 32) {
       const int j = j0 + lane;
       const bool in = j < n;
-      const uint32_t key = in ? ks[j] : 0u;
+      const uint32_t key = in ? ks[j] - kmin : 0u;
       const bool eq = in && key == T, gt = in && key > T;
       const unsigned em = __ballot_sync(FULL, eq);
       bool keep = gt || (eq && ties_seen + __popc(em & lt) < need);
@@ -907,7 +936,7 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
 }
 
 inline size_t select_smem_bytes(const Shape& sh) {
-  return sizeof(float) * ((size_t)SEL_R * sh.ld_scores + (size_t)SEL_R * 512);
+  return sizeof(float) * ((size_t)SEL_R * sh.ld_scores + (size_t)SEL_R * (sh.mode == 1 ? SEL_WARP_WORDS : SEL_WARP_WORDS - 512));
 }
 
 }  // namespace
@@ -959,7 +988,7 @@ cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws
 
 cudaError_t launch_choose(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
                           const ForcedPack& forced, int have_sics, cudaStream_t s) {
-  k_choose<<<sh.BH, 32, 0, s>>>(sh, gp, st, ws, forced, have_sics);
+  k_choose<<<sh.BH, 256, 0, s>>>(sh, gp, st, ws, forced, have_sics);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   k_groups<<<1, 1024, 0, s>>>(sh, gp, ws, 0);
