@@ -37,6 +37,12 @@
  *   - Every function returns SPADE_OK (0) or a negative spade_error_t; arguments are validated
  *     before anything is launched; nothing aborts.  spade_last_error() gives the message.
  *   - There is no CPU path: without a CUDA device every stage returns SPADE_ERR_CUDA.
+ *   - Debug build (compile the sources with -DSPADE_DEBUG; the Python binding loads it when the environment
+ *     has SPADE_DEBUG=1): every index a kernel takes from an index list, a histogram or a table is checked
+ *     before use.  A failed check never traps or faults: it is counted in the status words with the site and
+ *     the offending value, the access is skipped, and spade_status returns SPADE_ERR_DEBUG_CHECK.  The
+ *     workspace then also carries a 256-byte guard word behind every region (spade_workspace_bytes grows
+ *     accordingly), written by spade_plan and verified by spade_status.
  */
 #ifndef SPADE_H_
 #define SPADE_H_
@@ -55,7 +61,9 @@ typedef enum {
   SPADE_ERR_WORKSPACE = -3,       /* workspace pointer null or misaligned */
   SPADE_ERR_CUDA = -4,            /* a CUDA runtime / driver call failed (message holds the CUDA error) */
   SPADE_ERR_DEVICE_TIMEOUT = -5,  /* a bounded device-side wait ran out (reported by spade_status) */
-  SPADE_ERR_ORDER = -6            /* stage called before the stage it depends on */
+  SPADE_ERR_ORDER = -6,           /* stage called before the stage it depends on */
+  SPADE_ERR_DEBUG_CHECK = -7      /* debug build only: an index check inside a kernel failed, or a guard word behind a
+                                     workspace region was overwritten (reported by spade_status) */
 } spade_error_t;
 
 typedef struct spade_plan_s spade_plan_t;   /* opaque; created and destroyed by the library */

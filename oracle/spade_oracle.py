@@ -17,6 +17,9 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "spade_oracle.cpp")
 _LIB = os.path.join(_HERE, "libspade_oracle.so")
+_SANITIZE = os.environ.get("SPADE_ORACLE_SANITIZE") == "1"     # AddressSanitizer + UBSan build (run under LD_PRELOAD=libasan)
+if _SANITIZE:
+    _LIB = os.path.join(_HERE, "libspade_oracle_san.so")
 _lib = None
 
 _I = C.POINTER(C.c_int)
@@ -27,7 +30,8 @@ def build(force: bool = False) -> str:
     """Compile the oracle (g++ -O2, no fast-math: fp64 with the order the source states)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + f".tmp{os.getpid()}"
-        subprocess.check_call(["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread",
+        san = ["-fsanitize=address,undefined", "-fno-sanitize-recover=undefined", "-g", "-O1"] if _SANITIZE else ["-O2"]
+        subprocess.check_call(["g++"] + san + ["-std=c++17", "-fPIC", "-shared", "-pthread",
                                "-ffp-contract=off", _SRC, "-o", tmp])
         os.replace(tmp, _LIB)
     return _LIB

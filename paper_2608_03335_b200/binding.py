@@ -12,14 +12,14 @@ from typing import Dict, Optional, Sequence
 
 import torch
 
-from .build import LIB
+from .build import LIB, LIB_DEBUG, build_library
 
 SPADE_TOPK, SPADE_TOPP, SPADE_SPARSITY, SPADE_POLICY_AS = 0, 1, 2, 3
 ESTIMATORS = {"mean": 0, "dsa": 1, "dsa2": 2}       # spade_estimator_t
 MODES = {"topk": SPADE_TOPK, "topp": SPADE_TOPP, "sparsity": SPADE_SPARSITY, "policy_as": SPADE_POLICY_AS}
 
 ERRORS = {0: "SPADE_OK", -1: "SPADE_ERR_INVALID_ARG", -2: "SPADE_ERR_UNSUPPORTED", -3: "SPADE_ERR_WORKSPACE",
-          -4: "SPADE_ERR_CUDA", -5: "SPADE_ERR_DEVICE_TIMEOUT", -6: "SPADE_ERR_ORDER"}
+          -4: "SPADE_ERR_CUDA", -5: "SPADE_ERR_DEVICE_TIMEOUT", -6: "SPADE_ERR_ORDER", -7: "SPADE_ERR_DEBUG_CHECK"}
 
 
 class SpadeError(RuntimeError):
@@ -60,10 +60,13 @@ def lib():
     """Load libspade_b200.so (built in-tree by paper_2608_03335_b200.build); raise if absent."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB):
-            raise RuntimeError(f"{LIB} is missing: build it with `python -m paper_2608_03335_b200.build` "
+        path = LIB
+        if os.environ.get("SPADE_DEBUG") == "1":          # the checked build of the same kernels (see spade.h)
+            path = build_library(debug=True)
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: build it with `python -m paper_2608_03335_b200.build` "
                                "(there is no CPU fallback)")
-        L = C.CDLL(LIB)
+        L = C.CDLL(path)
         L.spade_last_error.restype = C.c_char_p
         L.spade_workspace_bytes.restype = C.c_size_t
         L.spade_workspace_bytes.argtypes = [C.c_void_p]

@@ -48,6 +48,8 @@ struct DeviceGuard {
 struct WsLayout {
   size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, nsum, scores, colkeep, rowfull, pair_axis, pair_union, mm, text_start, head_work, att_scratch;
   size_t bytes;
+  size_t canary[40];     // debug build: offsets of the 256-byte guard words after each region
+  int n_canary;
 };
 
 }  // namespace
@@ -136,7 +138,16 @@ void compute_layout(spade_plan_s* p) {
   sh.cap = sh.masks_on ? ((sh.NBmax + 3) & ~3) : p->base_cap;
   WsLayout& l = p->lay;
   size_t o = 0;
-  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+  l.n_canary = 0;
+  auto take = [&](size_t bytes) {
+    size_t at = o;
+    o = align_up(o + bytes, 256);
+#ifdef SPADE_DEBUG
+    if (l.n_canary < 40) l.canary[l.n_canary++] = o;       // a guard word behind every region
+    o += 256;
+#endif
+    return at;
+  };
   l.status = take(64 * 4);
   l.scheme = take((size_t)BH * 4);
   l.keep = take((size_t)BH * 4);
@@ -230,13 +241,13 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
     g.bt = cands[c].bt; g.bh = cands[c].bh; g.bw = cands[c].bw;
     if (g.bt < 1 || g.bh < 1 || g.bw < 1) { free(p); return fail(SPADE_ERR_INVALID_ARG, "candidate %d has a non-positive extent", c); }
     g.BS = g.bt * g.bh * g.bw;
-    if (g.BS != 64 && g.BS != 128) { free(p); return fail(SPADE_ERR_UNSUPPORTED, "candidate %d has %d tokens per block (64 or 128 needed)", c, g.BS); }
+    if (g.BS != 64 && g.BS != 128) { const int bs = g.BS; free(p); return fail(SPADE_ERR_UNSUPPORTED, "candidate %d has %d tokens per block (64 or 128 needed)", c, bs); }
     if (g.bt > 128 || g.bh > 128 || g.bw > 128) { free(p); return fail(SPADE_ERR_UNSUPPORTED, "candidate %d: extent above 128", c); }
     g.nbt = (sh.T + g.bt - 1) / g.bt; g.nbh = (sh.H + g.bh - 1) / g.bh; g.nbw = (sh.W + g.bw - 1) / g.bw;
     g.NBv = g.nbt * g.nbh * g.nbw;
     g.NBt = (sh.n_text + g.BS - 1) / g.BS;
     g.NB = g.NBv + g.NBt;
-    if (g.NB > SPADE_MAX_NB) { free(p); return fail(SPADE_ERR_UNSUPPORTED, "candidate %d gives %d blocks per head (max %d)", c, g.NB, SPADE_MAX_NB); }
+    if (g.NB > SPADE_MAX_NB) { const int nb = g.NB; free(p); return fail(SPADE_ERR_UNSUPPORTED, "candidate %d gives %d blocks per head (max %d)", c, nb, SPADE_MAX_NB); }
     g.pair = g.BS == 64;
     g.vtiles[0] = (g.nbt + 1) / 2 * g.nbh * g.nbw;
     g.vtiles[1] = g.nbt * ((g.nbh + 1) / 2) * g.nbw;
@@ -445,6 +456,9 @@ int spade_plan(spade_plan_t* p, const void* Q, const void* K, void* ws, void* st
   WsTables t = tables_at(p, ws);
   p->launches = 0;
   if (!p->keep_status) CUDA_TRY(cudaMemsetAsync(t.status, 0, 64 * 4, s));
+#ifdef SPADE_DEBUG
+  for (int i = 0; i < p->lay.n_canary; ++i) CUDA_TRY(cudaMemsetAsync((char*)ws + p->lay.canary[i], 0xC5, 256, s));
+#endif
   const bool skip_sics = forced != nullptr && !(p->sh.masks_on && p->sh.intra_thr > 0.f) && p->sh.mode != SPADE_POLICY_AS;
   // The caller's array is read here and never again: the schemes travel inside the launch itself
   // (4 bits per head), so a captured launch replays the values it was captured with.
@@ -650,6 +664,25 @@ int spade_status(spade_plan_t* p, void* ws, void* stream) {
   if (st[0] == SPADE_ST_TIMEOUT)
     return fail(SPADE_ERR_DEVICE_TIMEOUT, "a device-side wait gave up (site %u, work item %u)", st[1], st[2]);
   if (st[0] != 0) return fail(SPADE_ERR_CUDA, "device status %u", st[0]);
+#ifdef SPADE_DEBUG
+  {
+    uint32_t dbg[4] = {0, 0, 0, 0};
+    CUDA_TRY(cudaMemcpyAsync(dbg, tables_at(p, ws).status + 4, sizeof(dbg), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    if (dbg[0] != 0)
+      return fail(SPADE_ERR_DEBUG_CHECK, "%u index checks failed; first at site %u with value %u", dbg[0], dbg[1], dbg[2]);
+    if (p->stage > 0 && p->stage_ws == ws) {               // the workspace is laid out as this plan describes
+      std::vector<unsigned char> guard((size_t)p->lay.n_canary * 256);
+      for (int i = 0; i < p->lay.n_canary; ++i)
+        CUDA_TRY(cudaMemcpyAsync(guard.data() + (size_t)i * 256, (const char*)ws + p->lay.canary[i], 256, cudaMemcpyDeviceToHost,
+                                 (cudaStream_t)stream));
+      CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+      for (size_t i = 0; i < guard.size(); ++i)
+        if (guard[i] != 0xC5)
+          return fail(SPADE_ERR_DEBUG_CHECK, "guard word behind workspace region %zu was overwritten (byte %zu)", i / 256, i % 256);
+    }
+  }
+#endif
   return SPADE_OK;
 }
 

@@ -265,6 +265,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
           const int* row1 = ws.kv_idx + ((size_t)bh * sh.NBmax + (qb1 >= 0 ? qb1 : qb0)) * sh.cap;
           int cnt0 = ws.kv_cnt[(size_t)bh * sh.NBmax + qb0];
           int cnt1 = qb1 >= 0 ? ws.kv_cnt[(size_t)bh * sh.NBmax + qb1] : 0;
+          (void)SPADE_CHECK(cnt0 >= 0 && cnt0 <= sh.cap && cnt1 >= 0 && cnt1 <= sh.cap, ws.status, 403, cnt0);
           cnt0 = cnt0 < 0 ? 0 : (cnt0 > sh.cap ? sh.cap : cnt0);
           cnt1 = cnt1 < 0 ? 0 : (cnt1 > sh.cap ? sh.cap : cnt1);
           const int cmax = cnt0 > cnt1 ? cnt0 : cnt1;
@@ -297,7 +298,8 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
             while (u) {
               const int bit = __ffs(u) - 1;
               u &= u - 1;
-              list[pos] = (uint32_t)(wi * 32 + bit) | (((wa >> bit) & 1u) << 16) | (((wb >> bit) & 1u) << 17);
+              if (SPADE_CHECK(pos < SPADE_MAX_NB && wi * 32 + bit < g.NB, ws.status, 401, pos))
+                list[pos] = (uint32_t)(wi * 32 + bit) | (((wa >> bit) & 1u) << 16) | (((wb >> bit) & 1u) << 17);
               ++pos;
             }
           }
@@ -305,10 +307,12 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
         } else {
           const int* row = ws.kv_idx + ((size_t)bh * sh.NBmax + qb0) * sh.cap;
           int cnt = ws.kv_cnt[(size_t)bh * sh.NBmax + qb0];
+          (void)SPADE_CHECK(cnt >= 0 && cnt <= sh.cap, ws.status, 404, cnt);
           cnt = cnt < 0 ? 0 : (cnt > sh.cap ? sh.cap : cnt);
           cnt = cnt > SPADE_MAX_NB ? SPADE_MAX_NB : cnt;
           for (int e = lane; e < cnt; e += 32) {
             int id = row[e];
+            (void)SPADE_CHECK(id >= 0 && id < g.NB, ws.status, 402, id);
             list[e] = (uint32_t)((id >= 0 && id < g.NB) ? id : 0) | (3u << 16);
           }
           n_entries = cnt;
@@ -331,6 +335,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
           uint32_t e_next = H > 0 ? __ldcg(list) : 0u;
           for (int j = 0; j < H && !site; ++j, ++hc) {
             const int blk = (int)(e_next & 0xffffu);
+            (void)SPADE_CHECK(blk < g.NB, ws.status, 405, blk);
             const int half = g.pair ? 0 : (j & 1);
             const int jn = j + 1 < H ? j + 1 : j;
             e_next = __ldcg(list + (g.pair ? jn : (jn >> 1)));          // fetched one unit ahead

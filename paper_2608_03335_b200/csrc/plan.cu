@@ -58,12 +58,6 @@ __host__ __device__ constexpr uint32_t pf_idesc(int M, int N) {      // bf16 x b
   return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-// Valid tokens of block (it, ih, iw): edge blocks are partial.
-__device__ __forceinline__ float pf_inv_count(const Shape& sh, const CandGeo& g, int it, int ih, int iw) {
-  const int nt = min(g.bt, sh.T - it * g.bt), nh = min(g.bh, sh.H - ih * g.bh), nw = min(g.bw, sh.W - iw * g.bw);
-  return 1.f / (float)(nt * nh * nw);
-}
-
 __device__ __forceinline__ uint16_t pf_bf16(float x) {
   return __bfloat16_as_ushort(__float2bfloat16_rn(x));
 }
@@ -237,6 +231,7 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
 #pragma unroll
         for (int c = 0; c < 4; ++c) {                                    // the first four candidates: offsets kept in registers
           if (c >= sh.C) break;
+          if (!SPADE_CHECK(woff[c][2] < (uint32_t)W_BYTES && woff[c][0] < (uint32_t)W_BYTES, ws.status, 602, woff[c][0])) continue;
           *reinterpret_cast<uint16_t*>(wb + woff[c][0]) = r1;
           *reinterpret_cast<uint16_t*>(wb + woff[c][1]) = r2;
           *reinterpret_cast<uint16_t*>(wb + woff[c][2]) = r3;
@@ -304,7 +299,6 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
       uint32_t i = 0;
       for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
         const int col = item % col_items, chunk = (item / col_items) % cfg.nchunks, ht = item / (col_items * cfg.nchunks);
-        const int ch0 = (col / cfg.ncol_w) * cfg.colH, cw0 = (col % cfg.ncol_w) * cfg.colW;
         const int t0 = chunk * cfg.tchunk, t1 = min(sh.T, t0 + cfg.tchunk);
         for (int t = t0; t < t1 && !site; ++t, ++i) {
           const uint32_t b = i & 1, ph = (i >> 1) & 1;
@@ -337,7 +331,7 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
                 const int k = k4 + u;
-                if (e[u] >= 0) {
+                if (e[u] >= 0 && SPADE_CHECK(e[u] < sh.C * sh.NBmax, ws.status, 601, e[u])) {
                   cs[(size_t)e[u] * SPADE_D] = ar[k] * iv[u];          // mean summary, this channel
                   ns[(size_t)e[u] * SPADE_D] = an[k];                  // sum of q / |q|; SICS = its squared norm
                 }

@@ -201,6 +201,7 @@ k_blocks(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ 
         if (c_h0 + dh >= sh.nch) break;
         const int rowc = ((c_t0 + dt) * sh.nch + c_h0 + dh) * sh.ncw + c_w0;
         for (int dw = 0; dw < n_w && c_w0 + dw < sh.ncw; ++dw) {
+          if (!SPADE_CHECK(rowc + dw < sh.NCELL, ws.status, 501, rowc + dw)) continue;
           const float* p = cell0 + (size_t)(rowc + dw) * 2 * SPADE_D;
           const float4 a = *reinterpret_cast<const float4*>(p);
           const float4 r = *reinterpret_cast<const float4*>(p + SPADE_D);
@@ -776,7 +777,8 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
   int* out = ws.kv_idx + ((size_t)bh * sh.NBmax + row) * sh.cap;
   int count = 0;
   if (row >= n) {                               // text query block: every block
-    for (int j = lane; j < g.NB; j += 32) out[j] = j;
+    for (int j = lane; j < g.NB; j += 32)
+      if (SPADE_CHECK(j < sh.cap, ws.status, 301, j)) out[j] = j;
     if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = g.NB;
     return;
   }
@@ -819,7 +821,7 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
       const uint32_t key = j < n ? ks[j] - kmin : 0u;
       const bool hit = j < n && (key >> hi) == (T >> hi);
       const unsigned bm = __ballot_sync(FULL, hit);
-      if (hit) cand[at + __popc(bm & lt)] = key;
+      if (hit && SPADE_CHECK(at + __popc(bm & lt) < SEL_CAND, ws.status, 305, at)) cand[at + __popc(bm & lt)] = key;
       at += __popc(bm);
     }
     m = at;
@@ -839,7 +841,8 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
       const uint32_t base = m < 0 ? kmin : 0u;                     // the candidate list holds rel already
       for (int j = lane; j < cnt_all; j += 32) {
         const uint32_t key = src[j] - base;
-        if (hi >= 32 || (key >> hi) == (T >> hi)) atomicAdd(&hcnt[(key >> lo) & bmask], 1);
+        if ((hi >= 32 || (key >> hi) == (T >> hi)) && SPADE_CHECK(((key >> lo) & bmask) < 256u, ws.status, 304, (key >> lo) & bmask))
+          atomicAdd(&hcnt[(key >> lo) & bmask], 1);
       }
       __syncwarp();
       int above = 0;
@@ -907,7 +910,8 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
   if (sh.masks_on && ws.rowfull[(size_t)bh * sh.NBmax + row]) all = true;
   const int r_w = row % g.nbw, r_h = (row / g.nbw) % g.nbh, r_t = row / (g.nbw * g.nbh);
   if (all) {
-    for (int j = lane; j < n; j += 32) out[j] = j;
+    for (int j = lane; j < n; j += 32)
+      if (SPADE_CHECK(j < sh.cap, ws.status, 302, j)) out[j] = j;
     count = n;
   } else {
     int ties_seen = 0;
@@ -926,12 +930,13 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
         }
       }
       const unsigned km = __ballot_sync(FULL, keep);
-      if (keep) out[count + __popc(km & lt)] = j;
+      if (keep && SPADE_CHECK(count + __popc(km & lt) < sh.cap, ws.status, 303, count)) out[count + __popc(km & lt)] = j;
       count += __popc(km);
       ties_seen += __popc(em);
     }
   }
-  for (int j = lane; j < g.NBt; j += 32) out[count + j] = n + j;     // text KV blocks are always kept
+  for (int j = lane; j < g.NBt; j += 32)
+    if (SPADE_CHECK(count + j < sh.cap, ws.status, 306, count + j)) out[count + j] = n + j;     // text KV blocks are always kept
   if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt;
 }
 

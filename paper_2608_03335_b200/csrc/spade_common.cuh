@@ -103,6 +103,21 @@ enum : uint32_t {
   SPADE_ST_OK = 0,
   SPADE_ST_TIMEOUT = 1,     // status[0]: a bounded wait gave up; status[1] = where, status[2] = item
 };
+// Status words: [0..2] as above, [4] number of failed index checks of the debug build, [5] site of the first
+// one, [6] the offending value, [8] work-item counter of the attention kernel.
+
+// Debug build (-DSPADE_DEBUG): every index taken from a list, a histogram or a table is checked before use.
+// A failed check never traps: it is counted in the status words, the first site and value are kept, and the
+// access is skipped; spade_status reports it.  In the release build the macro is the constant `true`.
+#ifdef SPADE_DEBUG
+__device__ __forceinline__ bool spade_dbg_check(bool ok, uint32_t* status, uint32_t site, uint32_t value) {
+  if (!ok && atomicAdd(status + 4, 1u) == 0u) { status[5] = site; status[6] = value; }
+  return ok;
+}
+#define SPADE_CHECK(cond, status, site, value) spade_dbg_check((cond), (status), (site), (uint32_t)(value))
+#else
+#define SPADE_CHECK(cond, status, site, value) (true)
+#endif
 
 // Configuration of the one-pass scheme-generation kernel (plan.cu); on = 0 when the candidate set does not
 // fit it (a block footprint above 128 tokens in the (h, w) plane, more than 64 blocks of all candidates in one

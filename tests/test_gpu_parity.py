@@ -466,3 +466,48 @@ def test_policy_budget_follows_the_aggregation_score():
         pu.check_attention(w, plan, qb, kb, vb, O, scheme, rep)
     finally:
         plan.close()
+
+
+def test_topp_lists_are_reproducible_bit_for_bit_also_through_a_graph():
+    """The Top-P index search adds the softmax mass of a radix bin in fixed point, so the lists do not depend on
+    the order in which lanes reach a bin: two eager runs and two replays of a captured layer give identical
+    kv_idx / kv_cnt (and outputs)."""
+    from paper_2608_03335_b200 import binding
+    from paper_2608_03335_b200.workloads import make_qkv
+    w = small_variant(WORKLOADS["hunyuan"], heads=4, grid=(16, 18, 24), n_text=100)
+    Q, K, V = make_qkv(w, "cuda")
+    O = torch.empty_like(Q)
+    plan = binding.Plan(w.batch, w.heads, w.grid, w.n_text, w.candidates, w.mode, w.value)
+    try:
+        def layer(stream=None):
+            plan.spade_plan(Q, K, stream=stream)
+            plan.spade_summarize(Q, K, stream=stream)
+            plan.spade_select(stream=stream)
+            plan.spade_attn(Q, K, V, O, stream=stream)
+        runs = []
+        for _ in range(2):
+            layer()
+            torch.cuda.synchronize()
+            t = plan.tables()
+            runs.append((t["kv_idx"].clone(), t["kv_cnt"].clone(), O.clone()))
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(s):
+            with torch.cuda.graph(g, stream=s):
+                layer(stream=s)
+        for _ in range(2):
+            O.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            t = plan.tables()
+            runs.append((t["kv_idx"].clone(), t["kv_cnt"].clone(), O.clone()))
+        cnt0 = runs[0][1]
+        valid = torch.arange(runs[0][0].shape[2], device="cuda")[None, None, :] < cnt0[:, :, None]
+        for idx, cnt, out in runs[1:]:
+            assert torch.equal(cnt, cnt0)
+            assert torch.equal(idx[valid], runs[0][0][valid])
+            assert torch.equal(out, runs[0][2])
+        plan.spade_status()
+    finally:
+        plan.close()
