@@ -489,6 +489,24 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
         const bool all_valid = __all_sync(FULL, mask == ~0ull);
         if (!__all_sync(FULL, ptx::mbar_wait(&ctl.s_full, h & 1, &ctl.abort, WAIT_NS))) { site = 10; break; }
         ptx::tc_fence_after();
+        if (__all_sync(FULL, mask == 0ull)) {
+          // None of this warp's 32 rows takes part in the unit (the other half of a paired tile listed it, or the
+          // unit holds no real key): its weights are exact zeros, no score is read and no exponential is taken.
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&ctl.s_free);
+          if (!__all_sync(FULL, ptx::mbar_wait(&ctl.pv_done, (h & 1) ^ 1, &ctl.abort, WAIT_NS))) { site = 15; break; }
+          ptx::tc_fence_after();
+          uint32_t zero[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) zero[i] = 0u;
+          ptx::tmem_st32(tmem_P + lane_base, zero);
+          ptx::tmem_wait_st();
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&ctl.p_full);
+          continue;
+        }
         uint32_t sr[2][32];
         ptx::tmem_ld32(tmem_S + lane_base, sr[0]);
         ptx::tmem_ld32(tmem_S + lane_base + 32, sr[1]);
