@@ -46,7 +46,7 @@ struct DeviceGuard {
   CUDA_TRY(guard__.err)
 
 struct WsLayout {
-  size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, nsum, scores, colkeep, rowfull, pair_axis, pair_union, mm, text_start, head_work, att_scratch;
+  size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, ksplit, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, nsum, scores, colkeep, rowfull, pair_axis, pair_union, rowbits, mm, text_start, head_work, att_scratch;
   size_t bytes;
   size_t canary[40];     // debug build: offsets of the 256-byte guard words after each region
   int n_canary;
@@ -99,6 +99,7 @@ WsTables tables_at(const spade_plan_s* p, void* ws) {
   t.sics = (float*)(b + l.sics);
   t.qsum = (float*)(b + l.qsum);
   t.ksum = (float*)(b + l.ksum);
+  t.ksplit = (float*)(b + l.ksplit);
   t.kv_idx = (int*)(b + l.kv_idx);
   t.kv_cnt = (int*)(b + l.kv_cnt);
   t.head_order = (int*)(b + l.head_order);
@@ -112,6 +113,7 @@ WsTables tables_at(const spade_plan_s* p, void* ws) {
   t.scores = (float*)(b + l.scores);
   t.pair_axis = (int*)(b + l.pair_axis);
   t.pair_union = (int*)(b + l.pair_union);
+  t.rowbits = (uint32_t*)(b + l.rowbits);
   t.colkeep = (uint8_t*)(b + l.colkeep);
   t.rowfull = (uint8_t*)(b + l.rowfull);
   t.mm = (float*)(b + l.mm);
@@ -167,11 +169,14 @@ void compute_layout(spade_plan_s* p) {
   l.rowfull = take((size_t)BH * sh.NBmax);
   l.qsum = take((size_t)BH * sh.NBmax * SPADE_D * 4);
   l.ksum = take((size_t)BH * sh.NBmax * SPADE_D * 4);
+  l.ksplit = take((size_t)BH * 2 * sh.NBmax * SPADE_D * 4);
   l.kv_idx = take((size_t)BH * sh.NBmax * sh.cap * 4);
   l.cells = take(sh.use_cells && !p->pf.on ? (size_t)BH * 2 * sh.NCELL * 2 * SPADE_D * 4 : 0);
   l.csum = take(sh.use_cells || p->pf.on ? (size_t)BH * 2 * n_cands * sh.NBmax * SPADE_D * 4 : 0);
   l.nsum = take(p->pf.on ? (size_t)BH * 2 * n_cands * sh.NBmax * SPADE_D * 4 : 0);
   sh.ld_scores = (sh.NBvmax + 63) & ~63;
+  sh.bits_ld = sh.ld_scores / 32;
+  l.rowbits = take((size_t)BH * sh.NBvmax * sh.bits_ld * 4);
   l.scores = take((size_t)BH * sh.NBvmax * sh.ld_scores * 4);
   l.mm = take(sh.estimator ? (size_t)4 * BH * SPADE_D * sh.ld_scores * 4 : 0);
   l.att_scratch = take((size_t)2 * p->num_sms * 2 * SPADE_MAX_NB * 4);
@@ -509,6 +514,10 @@ int spade_summarize(spade_plan_t* p, const void* Q, const void* K, void* ws, voi
   if (p->have_csum) CUDA_TRY(launch_gather(p->sh, p->gp, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
   else CUDA_TRY(launch_summarize(Q, K, p->sh, p->gp, p->st, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
   p->launches += 1;
+  if (!p->sh.estimator) {
+    CUDA_TRY(launch_split_k(p->sh, p->gp, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
+    p->launches += 1;
+  }
   if (p->sh.estimator) {
     CUDA_TRY(launch_minmax(Q, K, p->sh, p->gp, p->st, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
     p->launches += 1;

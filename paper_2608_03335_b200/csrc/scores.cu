@@ -6,16 +6,16 @@
 // hi = x rounded to the nearest TF32 value and lo = x - hi (exact in fp32); the product uses the three terms
 // hi*hi + hi*lo + lo*hi (the dropped lo*lo term is at most 2^-22 relative, of either sign), all accumulated in one fp32
 // TMEM tile by tcgen05.mma kind::tf32.  A (128 query blocks x 128 channels, hi and lo) lives in TMEM,
-// B (64 KV blocks x 128 channels) arrives by TMA in two stages and is split in place in shared memory.
-// Warp 4 issues the TMA loads and the products; warps 0-3 stage A, split B and write the scores, so the
-// split of tile j+1 and the epilogue of tile j-1 run while the tensor pipe works on tile j.
+// B (64 KV blocks x 128 channels, hi and lo planes written by k_split_k) arrives by TMA through a ring of
+// stages.  Warp 4 issues the TMA loads and the products; warps 0-3 stage A and write the scores, so the
+// epilogue of tile j-1 runs while the tensor pipe works on tile j.
 #include <cuda.h>
 #include <stdio.h>
 
 #include "sm100_ptx.cuh"
 #include "spade_common.cuh"
 
-struct ScoreMaps { CUtensorMap k; };     // 3-D (128 floats, NBmax rows, head), box (32 floats, 64 rows, 1)
+struct ScoreMaps { CUtensorMap k; };     // 4-D (128 floats, NBmax rows, hi | lo, head), box (32 floats, 64 rows, 1, 1)
 
 namespace {
 
@@ -40,8 +40,7 @@ __device__ __forceinline__ void umma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, u
 }
 
 struct ScCtl {
-  uint64_t b_full[SC_NST]; // TMA landed a raw K' tile            (issuer -> compute warps)
-  uint64_t b_ready[SC_NST];// the tile is split into hi / lo      (compute warps -> issuer), 4 arrivals
+  uint64_t b_full[SC_NST]; // TMA landed a K' tile, hi and lo planes (copy engine -> issuer)
   uint64_t mma_done[2];    // products of the tile are complete   (issuer -> compute warps and itself)
   uint64_t d_free[2];      // the D tile has been read            (compute warps -> issuer), 4 arrivals
   uint64_t a_ready;        // A is staged in TMEM                 (compute warps -> issuer), 4 arrivals
@@ -59,7 +58,6 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
   if (tid == 0) {
     for (int b = 0; b < SC_NST; ++b) {
       ptx::mbar_init(&ctl.b_full[b], 1);
-      ptx::mbar_init(&ctl.b_ready[b], 4);
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl.mma_done[b], 1);
@@ -95,15 +93,16 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
         const uint32_t sB = ptx::smem_u32(smem);
         auto load_tile = [&](int ct) {                 // the stage of tile ct must be free
           const uint32_t st = (tiles_done + ct) % SC_NST;
-          ptx::mbar_expect_tx(&ctl.b_full[st], 4 * SC_SUB);
-          for (int s = 0; s < 4; ++s) ptx::tma_load_3d(smem + st * SC_STAGE + s * SC_SUB, &maps.k, &ctl.b_full[st], 32 * s, (ct0 + ct) * SC_N, bh);
+          ptx::mbar_expect_tx(&ctl.b_full[st], 8 * SC_SUB);
+          for (int s = 0; s < 8; ++s)       // four 32-channel sub-tiles of the hi plane, then of the lo plane
+            ptx::tma_load_4d(smem + st * SC_STAGE + s * SC_SUB, &maps.k, &ctl.b_full[st], 32 * (s & 3), (ct0 + ct) * SC_N, s >> 2, bh);
         };
         // every stage is free here: all products of the previous item were waited for below
         for (int ct = 0; ct < SC_NST && ct < n_ct; ++ct) load_tile(ct);
         if (!ptx::mbar_wait(&ctl.a_ready, items_done & 1, &ctl.abort, SC_WAIT_NS)) site = 101;
         for (int ct = 0; ct < n_ct && !site; ++ct) {
           const uint32_t t = tiles_done + ct, st = t % SC_NST, db = t & 1;
-          if (!ptx::mbar_wait(&ctl.b_ready[st], (t / SC_NST) & 1, &ctl.abort, SC_WAIT_NS) ||
+          if (!ptx::mbar_wait(&ctl.b_full[st], (t / SC_NST) & 1, &ctl.abort, SC_WAIT_NS) ||
               !ptx::mbar_wait(&ctl.d_free[db], ((t >> 1) & 1) ^ 1, &ctl.abort, SC_WAIT_NS)) { site = 102; break; }
           ptx::tc_fence_after();
           const uint32_t d = tm + 256 + db * SC_N;
@@ -160,25 +159,7 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
         if (lane == 0) ptx::mbar_arrive(&ctl.a_ready);
       }
       for (int ct = 0; ct <= n_ct && !site; ++ct) {
-        const uint32_t t = tiles_done + ct, st = t % SC_NST, par = (t / SC_NST) & 1;
-        if (ct < n_ct) {
-          // split B(ct) in place: the hi tile keeps the truncated values, the lo tile gets the remainders
-          if (!__all_sync(0xffffffffu, ptx::mbar_wait(&ctl.b_full[st], par, &ctl.abort, SC_WAIT_NS))) { site = 105; break; }
-          uint4* bh_ = reinterpret_cast<uint4*>(smem + st * SC_STAGE);
-          uint4* bl_ = reinterpret_cast<uint4*>(smem + st * SC_STAGE + 4 * SC_SUB);
-          for (int i = tid; i < 4 * SC_SUB / 16; i += 128) {
-            uint4 v = bh_[i], h, l;
-            h.x = (v.x + 0x1000u) & 0xffffe000u; l.x = __float_as_uint(__uint_as_float(v.x) - __uint_as_float(h.x));
-            h.y = (v.y + 0x1000u) & 0xffffe000u; l.y = __float_as_uint(__uint_as_float(v.y) - __uint_as_float(h.y));
-            h.z = (v.z + 0x1000u) & 0xffffe000u; l.z = __float_as_uint(__uint_as_float(v.z) - __uint_as_float(h.z));
-            h.w = (v.w + 0x1000u) & 0xffffe000u; l.w = __float_as_uint(__uint_as_float(v.w) - __uint_as_float(h.w));
-            bh_[i] = h;
-            bl_[i] = l;
-          }
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&ctl.b_ready[st]);
-        }
+        const uint32_t t = tiles_done + ct;
         if (ct >= 1) {
           // epilogue of tile ct-1 (the issuer is already on tile ct)
           const uint32_t tp = t - 1, sp = tp & 1;
@@ -237,11 +218,11 @@ size_t score_maps_bytes() { return sizeof(ScoreMaps); }
 int scores_encode_maps(ScoreMaps* out, const Shape& sh, const WsTables& ws, char* err, size_t errlen) {
   EncodeFn enc = encode_fn();
   if (!enc) { snprintf(err, errlen, "cuTensorMapEncodeTiled is not available from this driver"); return 1; }
-  const cuuint64_t dims[3] = {SPADE_D, (cuuint64_t)sh.NBmax, (cuuint64_t)sh.BH};
-  const cuuint64_t str[2] = {512, 512ull * sh.NBmax};
-  const cuuint32_t box[3] = {32, SC_N, 1};
-  const cuuint32_t es[3] = {1, 1, 1};
-  CUresult r = enc(&out->k, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, ws.ksum, dims, str, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  const cuuint64_t dims[4] = {SPADE_D, (cuuint64_t)sh.NBmax, 2, (cuuint64_t)sh.BH};
+  const cuuint64_t str[3] = {512, 512ull * sh.NBmax, 1024ull * sh.NBmax};
+  const cuuint32_t box[4] = {32, SC_N, 1, 1};
+  const cuuint32_t es[4] = {1, 1, 1, 1};
+  CUresult r = enc(&out->k, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ws.ksplit, dims, str, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (K' summaries) failed with %d", (int)r); return 1; }
   return 0;

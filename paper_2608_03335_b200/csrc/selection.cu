@@ -258,6 +258,27 @@ k_gather(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, W
   }
 }
 
+// K' of the chosen scheme, split for the tensor-core estimator (scores.cu): hi = the nearest TF32 value,
+// lo = the exact remainder, as two planes the estimator's TMA copies read directly.
+__global__ void __launch_bounds__(256)
+k_split_k(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws) {
+  const long total = (long)sh.BH * sh.NBmax * 32;          // float4 elements
+  for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
+    const int c4 = (int)(i & 31);
+    const long rowi = i >> 5;
+    const int b = (int)(rowi % sh.NBmax), bh = (int)(rowi / sh.NBmax);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (b < gp.g[ws.scheme[bh]].NBv) v = reinterpret_cast<const float4*>(ws.ksum + ((size_t)bh * sh.NBmax + b) * SPADE_D)[c4];
+    float4 h, l;
+    h.x = __uint_as_float((__float_as_uint(v.x) + 0x1000u) & 0xffffe000u); l.x = v.x - h.x;
+    h.y = __uint_as_float((__float_as_uint(v.y) + 0x1000u) & 0xffffe000u); l.y = v.y - h.y;
+    h.z = __uint_as_float((__float_as_uint(v.z) + 0x1000u) & 0xffffe000u); l.z = v.z - h.z;
+    h.w = __uint_as_float((__float_as_uint(v.w) + 0x1000u) & 0xffffe000u); l.w = v.w - h.w;
+    reinterpret_cast<float4*>(ws.ksplit + (((size_t)bh * 2 + 0) * sh.NBmax + b) * SPADE_D)[c4] = h;
+    reinterpret_cast<float4*>(ws.ksplit + (((size_t)bh * 2 + 1) * sh.NBmax + b) * SPADE_D)[c4] = l;
+  }
+}
+
 // One CTA per head: AS(X|c) = sum_b SICS (Eq. 3; fixed lane-strided order, one warp per (candidate, tensor)),
 // then warp 0: normalised score, argmax (ties -> lowest candidate) unless forced, and the head's keep count /
 // threshold.
@@ -399,7 +420,7 @@ __global__ void __launch_bounds__(1024) k_groups(const __grid_constant__ Shape s
 
 // Merged-list length of a head's query tiles for each pairing axis (on a sample of the blocks): one warp
 // per (head, axis, sampled video block with an even coordinate along the axis) adds |L_i u L_j| of the pair (or |L_i| of a lone
-// block).  The intersection is counted by binary search of L_i's entries in the ascending L_j.
+// block), read off the bitmaps of the lists that the index search leaves next to them.
 __global__ void __launch_bounds__(WARPS_PER_CTA * 32)
 k_pair_axis(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws) {
   const int lane = threadIdx.x & 31;
@@ -417,24 +438,16 @@ k_pair_axis(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp
     const int ca = axis == 2 ? cw : axis == 1 ? chh : ct;
     const int na = axis == 2 ? g.nbw : axis == 1 ? g.nbh : g.nbt;
     if (ca & 1) continue;
-    const int* Li = ws.kv_idx + ((size_t)bh * sh.NBmax + i) * sh.cap;
-    const int ni = ws.kv_cnt[(size_t)bh * sh.NBmax + i];
-    int uni = ni;
-    if (ca + 1 < na) {
-      const int j = i + (axis == 2 ? 1 : axis == 1 ? g.nbw : g.nbw * g.nbh);
-      const int* Lj = ws.kv_idx + ((size_t)bh * sh.NBmax + j) * sh.cap;
-      const int nj = ws.kv_cnt[(size_t)bh * sh.NBmax + j];
-      int common = 0;
-      for (int e = lane; e < ni; e += 32) {
-        const int v = Li[e];
-        int lo = 0, hi = nj;
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if (Lj[mid] < v) lo = mid + 1; else hi = mid; }
-        common += (lo < nj && Lj[lo] == v) ? 1 : 0;
-      }
+    // |L_i u L_j| over the video KV blocks = popcount of the OR of the two rows' bitmaps (the text blocks every
+    // list ends with are the same for all rows and do not change the ranking of the axes)
+    const uint32_t* Bi = ws.rowbits + ((size_t)bh * sh.NBvmax + i) * sh.bits_ld;
+    const int words = (g.NBv + 31) >> 5;
+    const uint32_t* Bj = Bi;
+    if (ca + 1 < na) Bj = Bi + (size_t)(axis == 2 ? 1 : axis == 1 ? g.nbw : g.nbw * g.nbh) * sh.bits_ld;
+    int uni = 0;
+    for (int wd = lane; wd < words; wd += 32) uni += __popc(Bi[wd] | Bj[wd]);
 #pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) common += __shfl_xor_sync(FULL, common, o);
-      uni = ni + nj - common;
-    }
+    for (int o = 16; o >= 1; o >>= 1) uni += __shfl_xor_sync(FULL, uni, o);
     if (lane == 0) atomicAdd(&ws.pair_union[bh * 3 + axis], uni);
   }
 }
@@ -909,9 +922,11 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
   const uint8_t* colkeep = ws.colkeep + (size_t)bh * sh.NBmax;
   if (sh.masks_on && ws.rowfull[(size_t)bh * sh.NBmax + row]) all = true;
   const int r_w = row % g.nbw, r_h = (row / g.nbw) % g.nbh, r_t = row / (g.nbw * g.nbh);
+  uint32_t* bits = ws.rowbits + ((size_t)bh * sh.NBvmax + row) * sh.bits_ld;      // the same list as a bitmap, for k_pair_axis
   if (all) {
     for (int j = lane; j < n; j += 32)
       if (SPADE_CHECK(j < sh.cap, ws.status, 302, j)) out[j] = j;
+    for (int wd = lane; wd * 32 < n; wd += 32) bits[wd] = n - wd * 32 >= 32 ? 0xffffffffu : (1u << (n - wd * 32)) - 1u;
     count = n;
   } else {
     int ties_seen = 0;
@@ -930,6 +945,7 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
         }
       }
       const unsigned km = __ballot_sync(FULL, keep);
+      if (lane == 0) bits[j0 >> 5] = km;
       if (keep && SPADE_CHECK(count + __popc(km & lt) < sh.cap, ws.status, 303, count)) out[count + __popc(km & lt)] = j;
       count += __popc(km);
       ties_seen += __popc(em);
@@ -988,6 +1004,14 @@ cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws
   long ctas = (total + 255) / 256;
   if (ctas > (long)num_sms * 16) ctas = (long)num_sms * 16;
   k_gather<<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_split_k(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s) {
+  const long total = (long)sh.BH * sh.NBmax * 32;
+  long ctas = (total + 255) / 256;
+  if (ctas > (long)num_sms * 16) ctas = (long)num_sms * 16;
+  k_split_k<<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
   return cudaGetLastError();
 }
 

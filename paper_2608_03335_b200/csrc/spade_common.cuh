@@ -45,6 +45,7 @@ struct Shape {
   int nct, nch, ncw, NCELL; // cells along each axis, cells per head
   int CS;                   // tokens per full cell
   int ld_scores;            // row length of the block-score scratch (NBvmax rounded up to 64)
+  int bits_ld;              // 32-bit words per row of the list bitmaps (ld_scores / 32)
   // static / intra-block masks united with the dynamic selection (masks_on = any of them enabled)
   int masks_on, window, sink;
   float intra_thr;
@@ -70,6 +71,7 @@ struct WsTables {
   float* sics;          // [BH][C][2][NBvmax]
   float* qsum;          // [BH][NBmax][128]
   float* ksum;          // [BH][NBmax][128]
+  float* ksplit;        // [BH][2][NBmax][128] K' split for the tensor-core estimator: nearest TF32 value, remainder
   int* kv_idx;          // [BH][NBmax][cap]
   int* kv_cnt;          // [BH][NBmax]
   int* head_order;      // [BH] order in which the attention kernel takes the heads
@@ -82,6 +84,7 @@ struct WsTables {
   float* nsum;          // same shape: sum over a block's tokens of q / |q| (one-pass scheme generation only)
   int* pair_axis;       // [BH] axis (0 t, 1 h, 2 w) along which 64-token query blocks are paired into 128-row tiles
   int* pair_union;      // [BH][3] total merged-list length for each pairing axis
+  uint32_t* rowbits;    // [BH][NBvmax][bits_ld] the video part of every video query block's list as a bitmap (bit j = KV block j kept)
   uint8_t* colkeep;     // [BH][NBmax] KV block kept by every query block (intra rule on K, sink)
   uint8_t* rowfull;     // [BH][NBmax] query block keeps every block (intra rule on Q)
   float* scores;        // [BH][NBvmax][ld_scores] block scores S = Q'K'^T / sqrt(d) of the chosen scheme
@@ -150,6 +153,7 @@ cudaError_t launch_blocks(const void* Q, const void* K, const Shape& sh, const G
                           const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_static(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws, cudaStream_t s);
 cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
+cudaError_t launch_split_k(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_choose(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
                           const ForcedPack& forced, int have_sics, cudaStream_t s);
 cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
