@@ -46,7 +46,7 @@ struct DeviceGuard {
   CUDA_TRY(guard__.err)
 
 struct WsLayout {
-  size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, ksplit, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, nsum, scores, colkeep, rowfull, pair_axis, pair_union, rowbits, mm, text_start, head_work, att_scratch;
+  size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, ksplit, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, nsum, scores, colkeep, rowfull, pair_axis, pair_union, rowbits, mm, qmid, kdsa, text_start, head_work, att_scratch;
   size_t bytes;
   size_t canary[40];     // debug build: offsets of the 256-byte guard words after each region
   int n_canary;
@@ -117,6 +117,8 @@ WsTables tables_at(const spade_plan_s* p, void* ws) {
   t.colkeep = (uint8_t*)(b + l.colkeep);
   t.rowfull = (uint8_t*)(b + l.rowfull);
   t.mm = (float*)(b + l.mm);
+  t.qmid = (float*)(b + l.qmid);
+  t.kdsa = (float*)(b + l.kdsa);
   t.att_scratch = (uint32_t*)(b + l.att_scratch);
   return t;
 }
@@ -179,6 +181,8 @@ void compute_layout(spade_plan_s* p) {
   l.rowbits = take((size_t)BH * sh.NBvmax * sh.bits_ld * 4);
   l.scores = take((size_t)BH * sh.NBvmax * sh.ld_scores * 4);
   l.mm = take(sh.estimator ? (size_t)4 * BH * SPADE_D * sh.ld_scores * 4 : 0);
+  l.qmid = take(sh.estimator == 1 ? (size_t)BH * sh.NBmax * SPADE_D * 4 : 0);
+  l.kdsa = take(sh.estimator == 1 ? (size_t)BH * 4 * sh.NBmax * SPADE_D * 4 : 0);
   l.att_scratch = take((size_t)2 * p->num_sms * 2 * SPADE_MAX_NB * 4);
   l.bytes = o;
 }
@@ -521,6 +525,10 @@ int spade_summarize(spade_plan_t* p, const void* Q, const void* K, void* ws, voi
   if (p->sh.estimator) {
     CUDA_TRY(launch_minmax(Q, K, p->sh, p->gp, p->st, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
     p->launches += 1;
+    if (p->sh.estimator == 1) {
+      CUDA_TRY(launch_dsa_rows(p->sh, p->gp, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
+      p->launches += 1;
+    }
   }
   p->stage = 2;
   return SPADE_OK;
@@ -532,7 +540,7 @@ int spade_select(spade_plan_t* p, void* ws, void* stream) {
   if (p->stage < 2 || p->stage_ws != ws) return fail(SPADE_ERR_ORDER, "spade_select needs spade_summarize on this workspace first");
   ON_PLAN_DEVICE(p);
   WsTables t = tables_at(p, ws);
-  if (p->sh.estimator) {
+  if (p->sh.estimator == 2) {
     CUDA_TRY(launch_scores_minmax(p->sh, p->gp, t, (cudaStream_t)stream));
   } else {
     if (p->smaps_ws != ws) {
@@ -540,7 +548,13 @@ int spade_select(spade_plan_t* p, void* ws, void* stream) {
       if (scores_encode_maps(p->smaps, p->sh, t, msg, sizeof(msg))) return fail(SPADE_ERR_CUDA, "tensor map: %s", msg);
       p->smaps_ws = ws;
     }
-    CUDA_TRY(launch_scores(p->smaps, p->sh, p->gp, t, p->num_sms, (cudaStream_t)stream));
+    if (p->sh.estimator == 1) {       // Fig. 4a as two tensor-core passes over the same score table
+      CUDA_TRY(launch_scores(p->smaps, p->sh, p->gp, t, p->num_sms, 1, (cudaStream_t)stream));
+      CUDA_TRY(launch_scores(p->smaps, p->sh, p->gp, t, p->num_sms, 2, (cudaStream_t)stream));
+      p->launches += 1;
+    } else {
+      CUDA_TRY(launch_scores(p->smaps, p->sh, p->gp, t, p->num_sms, 0, (cudaStream_t)stream));
+    }
   }
   CUDA_TRY(launch_select(p->sh, p->gp, p->st, t, (cudaStream_t)stream));
   p->launches += 2;

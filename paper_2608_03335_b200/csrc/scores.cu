@@ -15,7 +15,10 @@
 #include "sm100_ptx.cuh"
 #include "spade_common.cuh"
 
-struct ScoreMaps { CUtensorMap k; };     // 4-D (128 floats, NBmax rows, hi | lo, head), box (32 floats, 64 rows, 1, 1)
+struct ScoreMaps {
+  CUtensorMap k;      // 4-D (128 floats, NBmax rows, hi | lo, head) over the split K' means, box (32 floats, 64 rows, 1, 1)
+  CUtensorMap kd;     // same with four planes: hi | lo of k_mid, hi | lo of k_half (the max/min estimator of Fig. 4a)
+};
 
 namespace {
 
@@ -50,7 +53,11 @@ struct ScCtl {
 
 __global__ void __launch_bounds__(SC_THREADS, 1)
 k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp,
-         const WsTables ws, const float scale) {
+         const WsTables ws, const float scale, const float* __restrict__ a_rows, const int a_abs, const int term) {
+  // term 0: S = A K'^T with the mean summaries.  terms 1, 2: the two halves of the max/min estimator,
+  // S = q~ k_mid^T (written) and S += |q~| k_half^T (added to what term 1 left).
+  const CUtensorMap* const kmap = term == 0 ? &maps.k : &maps.kd;
+  const int plane0 = term == 2 ? 2 : 0;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   ScCtl& ctl = *reinterpret_cast<ScCtl*>(smem + SC_NST * SC_STAGE);
@@ -95,7 +102,7 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
           const uint32_t st = (tiles_done + ct) % SC_NST;
           ptx::mbar_expect_tx(&ctl.b_full[st], 8 * SC_SUB);
           for (int s = 0; s < 8; ++s)       // four 32-channel sub-tiles of the hi plane, then of the lo plane
-            ptx::tma_load_4d(smem + st * SC_STAGE + s * SC_SUB, &maps.k, &ctl.b_full[st], 32 * (s & 3), (ct0 + ct) * SC_N, s >> 2, bh);
+            ptx::tma_load_4d(smem + st * SC_STAGE + s * SC_SUB, kmap, &ctl.b_full[st], 32 * (s & 3), (ct0 + ct) * SC_N, plane0 + (s >> 2), bh);
         };
         // every stage is free here: all products of the previous item were waited for below
         for (int ct = 0; ct < SC_NST && ct < n_ct; ++ct) load_tile(ct);
@@ -135,13 +142,14 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
       const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
       const int row = rt * 128 + warp * 32 + lane;
       {
-        const float4* src = reinterpret_cast<const float4*>(ws.qsum + ((size_t)bh * sh.NBmax + (row < sh.NBmax ? row : 0)) * SPADE_D);
+        const float4* src = reinterpret_cast<const float4*>(a_rows + ((size_t)bh * sh.NBmax + (row < sh.NBmax ? row : 0)) * SPADE_D);
 #pragma unroll 1
         for (int ch = 0; ch < 4; ++ch) {
           uint32_t hi[32], lo[32];
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             float4 v = row < sh.NBmax ? __ldg(src + ch * 8 + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+            if (a_abs) { v.x = fabsf(v.x); v.y = fabsf(v.y); v.z = fabsf(v.z); v.w = fabsf(v.w); }
             const float x[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -173,10 +181,15 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
             ptx::tmem_wait_ld();
             if (row < nbv) {
 #pragma unroll
-              for (int q = 0; q < 8; ++q)
-                reinterpret_cast<float4*>(dst + ch * 32)[q] =
-                    make_float4(__uint_as_float(r[4 * q]) * scale, __uint_as_float(r[4 * q + 1]) * scale,
-                                __uint_as_float(r[4 * q + 2]) * scale, __uint_as_float(r[4 * q + 3]) * scale);
+              for (int q = 0; q < 8; ++q) {
+                float4 o = make_float4(__uint_as_float(r[4 * q]) * scale, __uint_as_float(r[4 * q + 1]) * scale,
+                                       __uint_as_float(r[4 * q + 2]) * scale, __uint_as_float(r[4 * q + 3]) * scale);
+                if (term == 2) {
+                  const float4 old = reinterpret_cast<const float4*>(dst + ch * 32)[q];
+                  o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                }
+                reinterpret_cast<float4*>(dst + ch * 32)[q] = o;
+              }
             }
           }
           ptx::tc_fence_before();
@@ -225,15 +238,23 @@ int scores_encode_maps(ScoreMaps* out, const Shape& sh, const WsTables& ws, char
   CUresult r = enc(&out->k, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ws.ksplit, dims, str, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (K' summaries) failed with %d", (int)r); return 1; }
+  if (sh.estimator == 1) {
+    const cuuint64_t dims4[4] = {SPADE_D, (cuuint64_t)sh.NBmax, 4, (cuuint64_t)sh.BH};
+    const cuuint64_t str4[3] = {512, 512ull * sh.NBmax, 2048ull * sh.NBmax};
+    r = enc(&out->kd, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, ws.kdsa, dims4, str4, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { snprintf(err, errlen, "cuTensorMapEncodeTiled (max/min summaries) failed with %d", (int)r); return 1; }
+  }
   return 0;
 }
 
 cudaError_t launch_scores(const ScoreMaps* maps, const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms,
-                          cudaStream_t s) {
+                          int term, cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(k_scores, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
   if (e != cudaSuccess) return e;
   const int items = sh.BH * ((sh.NBvmax + 127) / 128) * SC_PARTS;
   const int grid = items < num_sms ? items : num_sms;
-  k_scores<<<grid, SC_THREADS, SC_SMEM, s>>>(*maps, sh, gp, ws, 1.0f / sqrtf((float)SPADE_D));
+  k_scores<<<grid, SC_THREADS, SC_SMEM, s>>>(*maps, sh, gp, ws, 1.0f / sqrtf((float)SPADE_D), term == 0 ? ws.qsum : ws.qmid,
+                                             term == 2 ? 1 : 0, term);
   return cudaGetLastError();
 }

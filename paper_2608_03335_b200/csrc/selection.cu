@@ -258,6 +258,39 @@ k_gather(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, W
   }
 }
 
+// Max/min estimator of Fig. 4a on the tensor cores: S = q~ k_mid^T + |q~| k_half^T is a contraction over 256
+// channels.  The channel-major planes k_minmax leaves (what the SIMT estimator kernel reads) are turned into the
+// row-major operands of k_scores: q~ rows, and k_mid / k_half rows split into nearest TF32 value and remainder.
+// A CTA transposes a 32-channel x 32-block patch of one plane through shared memory.
+__global__ void __launch_bounds__(256)
+k_dsa_rows(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws) {
+  __shared__ float tile[32][33];
+  const int bh = blockIdx.z / 3, which = blockIdx.z % 3;            // 0: q~, 1: k_mid, 2: k_half
+  const int nbv = gp.g[ws.scheme[bh]].NBv;
+  const int b0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+  if (b0 >= ((nbv + 63) & ~63)) return;
+  const size_t plane = (size_t)sh.BH * SPADE_D * sh.ld_scores;
+  const float* src = ws.mm + (size_t)(which == 0 ? 0 : which + 1) * plane + ((size_t)bh * SPADE_D + c0) * sh.ld_scores + b0;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+#pragma unroll
+  for (int r = ty; r < 32; r += 8) tile[r][tx] = b0 + tx < sh.ld_scores ? src[(size_t)r * sh.ld_scores + tx] : 0.f;
+  __syncthreads();
+#pragma unroll
+  for (int r = ty; r < 32; r += 8) {
+    const int b = b0 + r;
+    if (b >= sh.NBmax) continue;
+    const float v = b < nbv ? tile[tx][r] : 0.f;
+    if (which == 0) {
+      ws.qmid[((size_t)bh * sh.NBmax + b) * SPADE_D + c0 + tx] = v;
+    } else {
+      const float h = __uint_as_float((__float_as_uint(v) + 0x1000u) & 0xffffe000u);
+      float* dst = ws.kdsa + (((size_t)bh * 4 + 2 * (which - 1)) * sh.NBmax + b) * SPADE_D + c0 + tx;
+      dst[0] = h;
+      dst[(size_t)sh.NBmax * SPADE_D] = v - h;
+    }
+  }
+}
+
 // K' of the chosen scheme, split for the tensor-core estimator (scores.cu): hi = the nearest TF32 value,
 // lo = the exact remainder, as two planes the estimator's TMA copies read directly.
 __global__ void __launch_bounds__(256)
@@ -1004,6 +1037,13 @@ cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws
   long ctas = (total + 255) / 256;
   if (ctas > (long)num_sms * 16) ctas = (long)num_sms * 16;
   k_gather<<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_dsa_rows(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s) {
+  (void)num_sms;
+  dim3 grid((sh.ld_scores + 31) / 32, SPADE_D / 32, sh.BH * 3);
+  k_dsa_rows<<<grid, 256, 0, s>>>(sh, gp, ws);
   return cudaGetLastError();
 }
 

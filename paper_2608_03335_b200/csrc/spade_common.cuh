@@ -90,6 +90,8 @@ struct WsTables {
   float* scores;        // [BH][NBvmax][ld_scores] block scores S = Q'K'^T / sqrt(d) of the chosen scheme
   uint32_t* att_scratch; // [2 * #SMs CTAs][2][SPADE_MAX_NB] merged index lists of the attention kernel's work items
   float* mm;            // [4][BH][128][ld_scores] channel-major max / min summaries (planes: see k_minmax)
+  float* qmid;          // [BH][NBmax][128] (q_max + q_min) / 2 row-major (SPADE_EST_DSA: operand A of the tensor-core estimator)
+  float* kdsa;          // [BH][4][NBmax][128] k_mid and k_half, each split into nearest TF32 value and remainder
 };
 
 struct GeoPack { CandGeo g[SPADE_MAX_CANDS]; };
@@ -181,7 +183,8 @@ struct ScoreMaps;  // tensor map of the K' summaries, defined in scores.cu
 size_t score_maps_bytes();
 int scores_encode_maps(ScoreMaps* out, const Shape& sh, const WsTables& ws, char* err, size_t errlen);
 cudaError_t launch_scores(const ScoreMaps* maps, const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms,
-                          cudaStream_t s);
+                          int term, cudaStream_t s);
+cudaError_t launch_dsa_rows(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
 
 struct AttnMaps;   // tensor maps of one (Q, K, V, O) quadruple, defined in attn.cu
 cudaError_t launch_attn(const AttnMaps* maps, const Shape& sh, const GeoPack& gp, const StaticTables& st,
