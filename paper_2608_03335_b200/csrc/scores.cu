@@ -38,7 +38,6 @@ constexpr int SC_ENTRY = 2 * SC_BOX;             // ring entry: two boxes (A: tw
 constexpr int SC_NST = 6;                        // ring entries
 constexpr int SC_OBUF = 32 * 128;                // staging buffer of one warp: 32 rows x 32 floats
 constexpr uint64_t SC_WAIT_NS = 2000000000ull;
-constexpr int SC_PARTS = 3;                      // work items per row tile (balance over the SMs)
 constexpr size_t SC_SMEM = SC_NST * SC_ENTRY + 8 * SC_OBUF + 1024 + 256;
 
 __host__ __device__ constexpr uint32_t idesc_tf32(int M, int N) {
@@ -60,24 +59,38 @@ struct ScCtl {
   uint64_t a_ready;        // A is split into TMEM                            (compute warps -> issuer), 4 arrivals
   uint32_t tmem_base;
   volatile uint32_t abort;
+  int seg_bh, seg_rem, seg_count;   // this CTA's range: first head, tile offset inside it, tiles
 };
 
-struct ScItem { int bh, rt, ct0, n_ct, nbv; };
+// The tiles of all heads form one sequence (head, row tile, column tile); CTA b takes the b-th of gridDim.x equal
+// ranges of it and walks its range in segments that stay inside one row tile (one A).
+struct ScSeg { int bh, rt, ct0, n_ct, nbv; };
+struct ScWalk { int bh, rt, ct, n, nbv, left; };
 
-// Work item -> (head, row tile, first column tile, column tiles); n_ct = 0 when the item is empty.
-__device__ __forceinline__ ScItem sc_item(int item, int row_tiles, const GeoPack& gp, const int* scheme) {
-  ScItem it;
-  const int part = item % SC_PARTS;
-  it.rt = (item / SC_PARTS) % row_tiles;
-  it.bh = item / (SC_PARTS * row_tiles);
-  it.nbv = gp.g[scheme[it.bh]].NBv;
-  it.ct0 = 0; it.n_ct = 0;
-  if (it.rt * 128 < it.nbv) {
-    const int n_ct_all = (it.nbv + SC_N - 1) / SC_N, per_part = (n_ct_all + SC_PARTS - 1) / SC_PARTS;
-    it.ct0 = part * per_part;
-    it.n_ct = max(0, min(per_part, n_ct_all - it.ct0));
+__device__ __forceinline__ int sc_side(const GeoPack& gp, const int* scheme, int bh) { return (gp.g[scheme[bh]].NBv + SC_N - 1) / SC_N; }
+
+__device__ __forceinline__ ScWalk sc_walk_init(int bh, int rem, int count, const GeoPack& gp, const int* scheme, int BH) {
+  ScWalk w;
+  w.bh = bh; w.left = count; w.nbv = 0; w.n = 0; w.rt = 0; w.ct = 0;
+  if (count > 0 && bh < BH) {
+    w.nbv = gp.g[scheme[bh]].NBv;
+    w.n = (w.nbv + SC_N - 1) / SC_N;
+    w.rt = rem / w.n; w.ct = rem % w.n;       // count > 0 puts the range's first tile inside this head: n > 0
   }
-  return it;
+  return w;
+}
+__device__ __forceinline__ bool sc_next(ScWalk& w, ScSeg& s, const GeoPack& gp, const int* scheme, int BH) {
+  if (w.left <= 0) return false;
+  while (w.rt >= w.n) {                        // on to the next head that has video blocks
+    if (++w.bh >= BH) return false;
+    w.nbv = gp.g[scheme[w.bh]].NBv;
+    w.n = (w.nbv + SC_N - 1) / SC_N; w.rt = 0; w.ct = 0;
+  }
+  s.bh = w.bh; s.rt = w.rt; s.ct0 = w.ct; s.nbv = w.nbv;
+  s.n_ct = min(w.left, w.n - w.ct);
+  w.left -= s.n_ct; w.ct += s.n_ct;
+  if (w.ct == w.n) { w.ct = 0; ++w.rt; }
+  return true;
 }
 
 __global__ void __launch_bounds__(SC_THREADS, 1)
@@ -107,25 +120,53 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
     ptx::fence_mbar_init();
   }
   if (warp == 4) { ptx::tmem_alloc(&ctl.tmem_base, 512); ptx::tmem_relinquish(); }
+  if (warp == 0) {
+    // tiles of all heads, then the head in which this CTA's range starts (warp scan over the heads, 32 at a time)
+    int total = 0;
+    for (int base = 0; base < sh.BH; base += 32) {
+      const int h = base + lane, n = h < sh.BH ? sc_side(gp, ws.scheme, h) : 0;
+      total += n * n;
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    const int lo = (int)((long long)blockIdx.x * total / gridDim.x), hi = (int)((long long)(blockIdx.x + 1) * total / gridDim.x);
+    int acc = 0, s_bh = sh.BH, s_rem = 0;
+    for (int base = 0; base < sh.BH && hi > lo; base += 32) {
+      const int h = base + lane, n = h < sh.BH ? sc_side(gp, ws.scheme, h) : 0;
+      int incl = n * n;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      const uint32_t hit = __ballot_sync(0xffffffffu, acc + incl > lo);
+      if (hit) {
+        const int first = __ffs(hit) - 1;
+        const int incl_f = __shfl_sync(0xffffffffu, incl, first), nn_f = __shfl_sync(0xffffffffu, n * n, first);
+        s_bh = base + first; s_rem = lo - (acc + incl_f - nn_f);
+        break;
+      }
+      acc += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) { ctl.seg_bh = s_bh; ctl.seg_rem = s_rem; ctl.seg_count = hi - lo; }
+  }
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tm = ctl.tmem_base;                 // A hi: cols 0..127, A lo: 128..255, D: 256..383 and 384..511
-  const int row_tiles = (sh.NBvmax + 127) / 128;
-  const int items = sh.BH * row_tiles * SC_PARTS;
+  ScWalk walk = sc_walk_init(ctl.seg_bh, ctl.seg_rem, ctl.seg_count, gp, ws.scheme, sh.BH);
+  ScSeg it;
   uint32_t ent = 0;                                   // ring entries so far (the same sequence in every role)
   uint32_t tiles = 0;                                 // column tiles so far
-  uint32_t items_done = 0;                            // non-empty items so far
+  uint32_t items_done = 0;                            // segments so far
   uint32_t site = 0;
   int site_item = 0;
 
   if (warp == 5) {
     // ================= loader: A rows and B slices by TMA, as far ahead as the ring allows ================
     if (lane == 0) {
-      for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
-        const ScItem it = sc_item(item, row_tiles, gp, ws.scheme);
-        if (it.n_ct == 0) continue;
-        site_item = item;
+      while (!site && sc_next(walk, it, gp, ws.scheme, sh.BH)) {
+        site_item = it.bh * 4096 + it.rt;
         for (int e = 0; e < 2 + 4 * it.n_ct; ++e, ++ent) {
           const uint32_t st = ent % SC_NST;
           if (!ptx::mbar_wait_sleepy(&ctl.empty[st], ((ent / SC_NST) & 1) ^ 1, &ctl.abort, SC_WAIT_NS)) { site = 101; break; }
@@ -153,10 +194,8 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
     if (lane == 0) {
       const uint32_t idesc = idesc_tf32(128, SC_N);
       const uint32_t sB = ptx::smem_u32(smem);
-      for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
-        const ScItem it = sc_item(item, row_tiles, gp, ws.scheme);
-        if (it.n_ct == 0) continue;
-        site_item = item;
+      while (!site && sc_next(walk, it, gp, ws.scheme, sh.BH)) {
+        site_item = it.bh * 4096 + it.rt;
         // the A entries are read by the compute warps; once A is in TMEM they go back to the loader
         if (!ptx::mbar_wait(&ctl.a_ready, items_done & 1, &ctl.abort, SC_WAIT_NS)) { site = 102; break; }
         ptx::mbar_arrive(&ctl.empty[ent % SC_NST]);
@@ -232,10 +271,8 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
       return true;
     };
 
-    for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
-      const ScItem it = sc_item(item, row_tiles, gp, ws.scheme);
-      if (it.n_ct == 0) continue;
-      site_item = item;
+    while (!site && sc_next(walk, it, gp, ws.scheme, sh.BH)) {
+      site_item = it.bh * 4096 + it.rt;
       // ---- A: this thread's row, 128 channels, from the two ring entries into TMEM as hi and lo --------------
       const uint32_t st0 = ent % SC_NST, st1 = (ent + 1) % SC_NST;
       if (!ptx::mbar_wait_warp(&ctl.full[st0], (ent / SC_NST) & 1, &ctl.abort, SC_WAIT_NS) ||
@@ -343,8 +380,9 @@ cudaError_t launch_scores(const ScoreMaps* maps, const Shape& sh, const GeoPack&
                           int term, cudaStream_t s) {
   cudaError_t e = cudaFuncSetAttribute(k_scores, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SC_SMEM);
   if (e != cudaSuccess) return e;
-  const int items = sh.BH * ((sh.NBvmax + 127) / 128) * SC_PARTS;
-  const int grid = items < num_sms ? items : num_sms;
+  const int side = (sh.NBvmax + SC_N - 1) / SC_N;
+  const long long most = (long long)sh.BH * side * side;       // tiles if every head took the finest candidate
+  const int grid = most < num_sms ? (int)(most > 0 ? most : 1) : num_sms;
   k_scores<<<grid, SC_THREADS, SC_SMEM, s>>>(*maps, sh, gp, ws, 1.0f / sqrtf((float)SPADE_D), term == 2 ? 1 : 0, term);
   return cudaGetLastError();
 }

@@ -989,6 +989,231 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
   if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt;
 }
 
+// Top-K index search with the row held in registers (rows of up to NV * 128 blocks): the same radix descent as
+// k_select, but the scores are read once into NV float4 per lane, turned into keys relative to the row's minimum
+// there, and the first histogram pass, the copy of the cut's bin into the candidate list and the final emit all
+// work from those registers.  Lane l holds blocks 128 u + 4 l .. + 3 of vector u, so a lane's four keep bits are
+// consecutive ids: list positions come from one warp scan per vector, the bitmap word from three shuffles.
+constexpr int SELR_WORDS = 296 + SEL_CAND;      // per warp: 256 bin counts, 32 dump slots, the list counter (word 288); candidate keys
+
+template <int NV>
+__global__ void __launch_bounds__(SEL_R * 32, 3)
+k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws) {
+  __shared__ int sel_sm[SEL_R * SELR_WORDS];
+  const int bh = blockIdx.y;
+  const CandGeo& g = gp.g[ws.scheme[bh]];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int row = blockIdx.x * SEL_R + warp;
+  if (row >= g.NB) return;
+  const int n = g.NBv;
+  int* out = ws.kv_idx + ((size_t)bh * sh.NBmax + row) * sh.cap;
+  if (row >= n) {                               // text query block: every block
+    for (int j = lane; j < g.NB; j += 32)
+      if (SPADE_CHECK(j < sh.cap, ws.status, 301, j)) out[j] = j;
+    if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = g.NB;
+    return;
+  }
+  int* hcnt = sel_sm + warp * SELR_WORDS;                        // [256] bins, [256 + lane] dump slots, [288] list counter
+  uint32_t* cand = reinterpret_cast<uint32_t*>(hcnt + 296);      // [SEL_CAND]
+  const int ldc = sh.ld_scores;
+
+  // ---- the row: NV float4 per lane, keys, range ---------------------------------------------------------
+  // Slots past the row's end take rel = 0, the row's minimum: they sit below (or tie with) every block and carry the
+  // highest ids, so neither the k-th largest value nor the choice among its ties (lowest ids first) changes.
+  uint32_t rel[NV][4];
+  {
+    const float4* src = reinterpret_cast<const float4*>(ws.scores + ((size_t)bh * sh.NBvmax + row) * ldc);
+    float4 v[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+      const int i = u * 32 + lane;
+      v[u] = 4 * i < n ? __ldcs(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);      // rows are ld_scores long (a multiple of 64)
+    }
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+      rel[u][0] = order_key(v[u].x); rel[u][1] = order_key(v[u].y); rel[u][2] = order_key(v[u].z); rel[u][3] = order_key(v[u].w);
+    }
+  }
+  uint32_t kmax = 0u, kmin = 0xffffffffu;
+#pragma unroll
+  for (int u = 0; u < NV; ++u) {
+    const int left = n - (u * 32 + lane) * 4;                    // valid keys of this vector: min(left, 4)
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (e < left) { kmax = max(kmax, rel[u][e]); kmin = min(kmin, rel[u][e]); }
+  }
+#pragma unroll
+  for (int o = 16; o >= 1; o >>= 1) {
+    kmax = max(kmax, __shfl_xor_sync(FULL, kmax, o));
+    kmin = min(kmin, __shfl_xor_sync(FULL, kmin, o));
+  }
+#pragma unroll
+  for (int u = 0; u < NV; ++u) {
+    const int left = n - (u * 32 + lane) * 4;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) rel[u][e] = e < left ? rel[u][e] - kmin : 0u;
+  }
+  const int n_pad = min(NV * 128, (n + 127) & ~127);             // slots the register passes count
+
+  // ---- radix descent on rel, from the top bit of the row's range down to bit 0 -----------------------------
+  int hi = kmax != kmin ? 32 - __clz(kmax - kmin) : 0;           // rel < 2^hi
+  uint32_t T = 0u;                                                // becomes rel of the last kept value
+  int need = ws.keep[bh];                                         // then: how many blocks with rel == T are kept (lowest ids first)
+  int cnt_T = n_pad;                                              // slots under the prefix found so far
+  bool all = need >= n;
+  int m = -1;                                                     // -1: the candidates are the row in registers; >= 0: cand[0 .. m)
+  while (hi > 0 && !all) {
+    const int lo = hi > 8 ? hi - 8 : 0;
+    const uint32_t bmask = (1u << (hi - lo)) - 1u;
+    for (int i = lane; i < 256; i += 32) hcnt[i] = 0;
+    __syncwarp();
+    if (m < 0) {
+      const uint32_t pre = __funnelshift_rc(T, 0u, hi);           // T >> hi, 0 when hi = 32
+#pragma unroll
+      for (int u = 0; u < NV; ++u) {
+        if (u * 128 >= n) break;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t key = rel[u][e];
+          const bool hit = __funnelshift_rc(key, 0u, hi) == pre;
+          atomicAdd(&hcnt[hit ? (key >> lo) & bmask : 256u + lane], 1);        // misses go to the lane's own dump slot
+        }
+      }
+    } else {
+      for (int j = lane; j < m; j += 32) {
+        const uint32_t key = cand[j];
+        if ((key >> hi) == (T >> hi)) atomicAdd(&hcnt[(key >> lo) & bmask], 1);
+      }
+    }
+    __syncwarp();
+    int above = 0;
+    const int bin = find_bin<int>(hcnt, need, above, lane);
+    if (bin < 0) { all = true; break; }          // cannot happen (need <= keys under the prefix); keep the row whole if it does
+    T |= (uint32_t)bin << lo;
+    need -= above;
+    hi = lo;
+    cnt_T = hcnt[bin];
+    __syncwarp();
+    if (m < 0 && hi > 0 && cnt_T <= SEL_CAND) {
+      // the bin the cut falls in is short: copy its keys out (in any order: the passes below only count them)
+      if (lane == 0) hcnt[288] = 0;
+      __syncwarp();
+      const uint32_t pre = T >> hi;
+#pragma unroll
+      for (int u = 0; u < NV; ++u) {
+        if (u * 128 >= n) break;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t key = rel[u][e];
+          if ((key >> hi) == pre) {
+            const int at = atomicAdd(&hcnt[288], 1);
+            if (SPADE_CHECK(at < SEL_CAND, ws.status, 305, at)) cand[at] = key;
+          }
+        }
+      }
+      m = cnt_T;
+      __syncwarp();
+    }
+  }
+
+  // ---- emit ascending ids (dynamic selection united with the static masks) ---------------------------------
+  const uint8_t* colkeep = ws.colkeep + (size_t)bh * sh.NBmax;
+  if (sh.masks_on && ws.rowfull[(size_t)bh * sh.NBmax + row]) all = true;
+  uint32_t* bits = ws.rowbits + ((size_t)bh * sh.NBvmax + row) * sh.bits_ld;      // the same list as a bitmap, for k_pair_axis
+  int count = 0;
+  if (all) {
+    for (int j = lane; j < n; j += 32)
+      if (SPADE_CHECK(j < sh.cap, ws.status, 302, j)) out[j] = j;
+    for (int wd = lane; wd * 32 < n; wd += 32) bits[wd] = n - wd * 32 >= 32 ? 0xffffffffu : (1u << (n - wd * 32)) - 1u;
+    count = n;
+  } else {
+    const bool ties = need < cnt_T;              // only some of the keys equal to T are kept: rank them by id
+    const int r_w = row % g.nbw, r_h = (row / g.nbw) % g.nbh, r_t = row / (g.nbw * g.nbh);
+    // The comparisons run over the registers once (straight-line code that every row executes a single time is
+    // bound by instruction fetch, so it is kept short); the keep bits of a lane's four blocks per vector are packed
+    // into one 64-bit word and the list is written by a rolled loop over the vectors.
+    unsigned long long knp = 0ull, eqp = 0ull;
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+      if (u * 128 >= n) break;
+      const int left = n - (u * 32 + lane) * 4;
+      uint32_t kn = 0u;
+      if (!ties) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) kn |= (e < left && rel[u][e] >= T ? 1u : 0u) << e;
+      } else {
+        uint32_t eqn = 0u;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          kn |= (e < left && rel[u][e] > T ? 1u : 0u) << e;
+          eqn |= (e < left && rel[u][e] == T ? 1u : 0u) << e;
+        }
+        eqp |= (unsigned long long)eqn << (4 * u);
+      }
+      knp |= (unsigned long long)kn << (4 * u);
+    }
+    int ties_seen = 0;
+    const int nvec = (n + 127) >> 7;
+#pragma unroll 1
+    for (int u = 0; u < nvec; ++u) {
+      const int j0 = (u * 32 + lane) * 4, left = n - j0;
+      uint32_t kn = (uint32_t)(knp >> (4 * u)) & 15u;      // keep bits of this lane's four blocks
+      if (ties) {
+        const uint32_t eqn = (uint32_t)(eqp >> (4 * u)) & 15u;
+        const int c = __popc(eqn);
+        int incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int up = __shfl_up_sync(FULL, incl, o);
+          if (lane >= o) incl += up;
+        }
+        int r = ties_seen + incl - c;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if ((eqn >> e) & 1u) { if (r < need) kn |= 1u << e; ++r; }
+        ties_seen += __shfl_sync(FULL, incl, 31);
+      }
+      if (sh.masks_on) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int j = j0 + e;
+          if (e < left) {
+            bool k = colkeep[j] != 0;
+            if (sh.window >= 0) {
+              const int dw = j % g.nbw - r_w, dh = (j / g.nbw) % g.nbh - r_h, dt = j / (g.nbw * g.nbh) - r_t;
+              k = k || (abs(dw) <= sh.window && abs(dh) <= sh.window && abs(dt) <= sh.window);
+            }
+            kn |= (k ? 1u : 0u) << e;
+          }
+        }
+      }
+      const int c = __popc(kn);
+      int incl = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(FULL, incl, o);
+        if (lane >= o) incl += up;
+      }
+      int pos = count + incl - c;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if ((kn >> e) & 1u) {
+          if (SPADE_CHECK(pos < sh.cap, ws.status, 303, pos)) out[pos] = j0 + e;
+          ++pos;
+        }
+      count += __shfl_sync(FULL, incl, 31);
+      uint32_t w = kn << (4 * (lane & 7));
+      w |= __shfl_xor_sync(FULL, w, 1);
+      w |= __shfl_xor_sync(FULL, w, 2);
+      w |= __shfl_xor_sync(FULL, w, 4);
+      if ((lane & 7) == 0 && (u * 4 + (lane >> 3)) * 32 < n) bits[u * 4 + (lane >> 3)] = w;
+    }
+  }
+  for (int j = lane; j < g.NBt; j += 32)
+    if (SPADE_CHECK(count + j < sh.cap, ws.status, 306, count + j)) out[count + j] = n + j;     // text KV blocks are always kept
+  if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt;
+}
+
 inline size_t select_smem_bytes(const Shape& sh) {
   return sizeof(float) * ((size_t)SEL_R * sh.ld_scores + (size_t)SEL_R * (sh.mode == 1 ? SEL_WARP_WORDS : SEL_WARP_WORDS - 512));
 }
@@ -1115,10 +1340,17 @@ cudaError_t launch_scores_minmax(const Shape& sh, const GeoPack& gp, const WsTab
 
 cudaError_t launch_select(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
                           cudaStream_t s) {
+  dim3 grid((sh.NBmax + SEL_R - 1) / SEL_R, sh.BH);
+  if (sh.mode != 1 && sh.NBvmax <= 16 * 128) {          // Top-K with rows that fit the register file
+    if (sh.NBvmax <= 4 * 128) k_select_topk<4><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else if (sh.NBvmax <= 8 * 128) k_select_topk<8><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else if (sh.NBvmax <= 12 * 128) k_select_topk<12><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else k_select_topk<16><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    return cudaGetLastError();
+  }
   const size_t smem = select_smem_bytes(sh);
   cudaError_t e = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  dim3 grid((sh.NBmax + SEL_R - 1) / SEL_R, sh.BH);
   k_select<<<grid, SEL_R * 32, smem, s>>>(sh, gp, st, ws);
   return cudaGetLastError();
 }
