@@ -989,12 +989,17 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
   if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt;
 }
 
-// Top-K index search with the row held in registers (rows of up to NV * 128 blocks): the same radix descent as
-// k_select, but the scores are read once into NV float4 per lane, turned into keys relative to the row's minimum
-// there, and the first histogram pass, the copy of the cut's bin into the candidate list and the final emit all
-// work from those registers.  Lane l holds blocks 128 u + 4 l .. + 3 of vector u, so a lane's four keep bits are
-// consecutive ids: list positions come from one warp scan per vector, the bitmap word from three shuffles.
-constexpr int SELR_WORDS = 296 + SEL_CAND;      // per warp: 256 bin counts, 32 dump slots, the list counter (word 288); candidate keys
+// Top-K index search with the row held in registers (rows of up to NV * 128 blocks).  The scores are read once
+// into NV float4 per lane.  The k-th largest value is found by histogram passes that are LINEAR in the value
+// between the smallest and largest score still in the race (250 bins), so that a row of roughly bell-shaped
+// scores leaves a dozen values in the bin the cut falls in; up to 64 of them are then ranked directly (every
+// lane counts how many are larger than its own).  A bin with more than 64 is split again between its own
+// minimum and maximum.  Binning only decides which values are ranked: the kept set is the exact top-k of the
+// fp32 scores, ties by lower id.  Lane l holds blocks 128 u + 4 l .. + 3 of vector u, so a lane's four keep bits
+// are consecutive ids: eight lanes' nibbles make a word of the row's bitmap, and the ascending id list is written
+// from the bitmap words.
+constexpr int SELR_CAND = 64;
+constexpr int SELR_WORDS = 296 + SELR_CAND + 64;   // per warp: 256 bin counts, 32 dump slots, list counter (word 288); candidates; bitmap words
 
 template <int NV>
 __global__ void __launch_bounds__(SEL_R * 32, 3)
@@ -1014,201 +1019,223 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
     return;
   }
   int* hcnt = sel_sm + warp * SELR_WORDS;                        // [256] bins, [256 + lane] dump slots, [288] list counter
-  uint32_t* cand = reinterpret_cast<uint32_t*>(hcnt + 296);      // [SEL_CAND]
+  float* cand = reinterpret_cast<float*>(hcnt + 296);            // [SELR_CAND]
+  uint32_t* words = reinterpret_cast<uint32_t*>(hcnt + 296 + SELR_CAND);     // [64] the row's keep bitmap
   const int ldc = sh.ld_scores;
 
-  // ---- the row: NV float4 per lane, keys, range ---------------------------------------------------------
-  // Slots past the row's end take rel = 0, the row's minimum: they sit below (or tie with) every block and carry the
-  // highest ids, so neither the k-th largest value nor the choice among its ties (lowest ids first) changes.
-  uint32_t rel[NV][4];
+  // ---- the row: NV float4 per lane; slots past the row's end hold NaN, which fails every comparison below ----------
+  float v[NV][4];
   {
     const float4* src = reinterpret_cast<const float4*>(ws.scores + ((size_t)bh * sh.NBvmax + row) * ldc);
-    float4 v[NV];
+    const float qnan = __int_as_float(0x7fffffff);
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
-      const int i = u * 32 + lane;
-      v[u] = 4 * i < n ? __ldcs(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);      // rows are ld_scores long (a multiple of 64)
-    }
-#pragma unroll
-    for (int u = 0; u < NV; ++u) {
-      rel[u][0] = order_key(v[u].x); rel[u][1] = order_key(v[u].y); rel[u][2] = order_key(v[u].z); rel[u][3] = order_key(v[u].w);
+      const int i = u * 32 + lane, left = n - 4 * i;
+      const float4 f = left > 0 ? __ldcs(src + i) : make_float4(qnan, qnan, qnan, qnan);      // rows are ld_scores long (a multiple of 64)
+      v[u][0] = f.x; v[u][1] = left > 1 ? f.y : qnan; v[u][2] = left > 2 ? f.z : qnan; v[u][3] = left > 3 ? f.w : qnan;
     }
   }
-  uint32_t kmax = 0u, kmin = 0xffffffffu;
+  float lo_v = INFINITY, hi_v = -INFINITY;
 #pragma unroll
-  for (int u = 0; u < NV; ++u) {
-    const int left = n - (u * 32 + lane) * 4;                    // valid keys of this vector: min(left, 4)
+  for (int u = 0; u < NV; ++u)
 #pragma unroll
-    for (int e = 0; e < 4; ++e)
-      if (e < left) { kmax = max(kmax, rel[u][e]); kmin = min(kmin, rel[u][e]); }
-  }
+    for (int e = 0; e < 4; ++e) { lo_v = fminf(lo_v, v[u][e]); hi_v = fmaxf(hi_v, v[u][e]); }     // NaN operands are ignored
 #pragma unroll
   for (int o = 16; o >= 1; o >>= 1) {
-    kmax = max(kmax, __shfl_xor_sync(FULL, kmax, o));
-    kmin = min(kmin, __shfl_xor_sync(FULL, kmin, o));
+    lo_v = fminf(lo_v, __shfl_xor_sync(FULL, lo_v, o));
+    hi_v = fmaxf(hi_v, __shfl_xor_sync(FULL, hi_v, o));
   }
-#pragma unroll
-  for (int u = 0; u < NV; ++u) {
-    const int left = n - (u * 32 + lane) * 4;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) rel[u][e] = e < left ? rel[u][e] - kmin : 0u;
-  }
-  const int n_pad = min(NV * 128, (n + 127) & ~127);             // slots the register passes count
 
-  // ---- radix descent on rel, from the top bit of the row's range down to bit 0 -----------------------------
-  int hi = kmax != kmin ? 32 - __clz(kmax - kmin) : 0;           // rel < 2^hi
-  uint32_t T = 0u;                                                // becomes rel of the last kept value
-  int need = ws.keep[bh];                                         // then: how many blocks with rel == T are kept (lowest ids first)
-  int cnt_T = n_pad;                                              // slots under the prefix found so far
-  bool all = need >= n;
-  int m = -1;                                                     // -1: the candidates are the row in registers; >= 0: cand[0 .. m)
-  while (hi > 0 && !all) {
-    const int lo = hi > 8 ? hi - 8 : 0;
-    const uint32_t bmask = (1u << (hi - lo)) - 1u;
+  // ---- the cut: keep v > T_hi, and need_t of the cnt_T blocks with T_lo <= v <= T_hi (lowest ids first) ---------------
+  int need_r = ws.keep[bh];                                       // blocks still to keep among those in [lo_v, hi_v]
+  bool all = need_r >= n;
+  int m = n;                                                      // blocks in [lo_v, hi_v]
+  float T_lo = 0.f, T_hi = 0.f;
+  int need_t = 0, cnt_T = 0;
+  for (int level = 0; !all; ++level) {
+    const float range = hi_v - lo_v;
+    if (!(range > 1e-30f) || level >= 40) {                       // one value left (or values no fp32 arithmetic tells apart): ties
+      T_lo = lo_v; T_hi = hi_v; need_t = need_r; cnt_T = m;
+      break;
+    }
+    const float a = 250.f / range;
     for (int i = lane; i < 256; i += 32) hcnt[i] = 0;
     __syncwarp();
-    if (m < 0) {
-      const uint32_t pre = __funnelshift_rc(T, 0u, hi);           // T >> hi, 0 when hi = 32
 #pragma unroll
-      for (int u = 0; u < NV; ++u) {
-        if (u * 128 >= n) break;
+    for (int u = 0; u < NV; ++u) {
+      if (u * 128 >= n) break;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const uint32_t key = rel[u][e];
-          const bool hit = __funnelshift_rc(key, 0u, hi) == pre;
-          atomicAdd(&hcnt[hit ? (key >> lo) & bmask : 256u + lane], 1);        // misses go to the lane's own dump slot
-        }
-      }
-    } else {
-      for (int j = lane; j < m; j += 32) {
-        const uint32_t key = cand[j];
-        if ((key >> hi) == (T >> hi)) atomicAdd(&hcnt[(key >> lo) & bmask], 1);
+      for (int e = 0; e < 4; ++e) {
+        const float d = v[u][e] - lo_v;
+        const bool in = d >= 0.f && d <= range;
+        const uint32_t bin = __float_as_uint(fmaf(d, a, 8388610.f)) & 255u;        // 2 .. 252, monotone in the value
+        atomicAdd(&hcnt[in ? bin : 256u + lane], 1);                             // misses go to the lane's own dump slot
       }
     }
     __syncwarp();
     int above = 0;
-    const int bin = find_bin<int>(hcnt, need, above, lane);
-    if (bin < 0) { all = true; break; }          // cannot happen (need <= keys under the prefix); keep the row whole if it does
-    T |= (uint32_t)bin << lo;
-    need -= above;
-    hi = lo;
-    cnt_T = hcnt[bin];
+    const int cut = find_bin<int>(hcnt, need_r, above, lane);
+    if (cut < 0) { all = true; break; }          // cannot happen (need_r <= blocks in range); keep the row whole if it does
+    need_r -= above;
+    m = hcnt[cut];
     __syncwarp();
-    if (m < 0 && hi > 0 && cnt_T <= SEL_CAND) {
-      // the bin the cut falls in is short: copy its keys out (in any order: the passes below only count them)
-      if (lane == 0) hcnt[288] = 0;
-      __syncwarp();
-      const uint32_t pre = T >> hi;
+    // one more pass over the registers: the cut bin's own range, and (when it is short) its values
+    const bool collect = m <= SELR_CAND;
+    if (lane == 0) hcnt[288] = 0;
+    __syncwarp();
+    float lo_n = INFINITY, hi_n = -INFINITY;
 #pragma unroll
-      for (int u = 0; u < NV; ++u) {
-        if (u * 128 >= n) break;
+    for (int u = 0; u < NV; ++u) {
+      if (u * 128 >= n) break;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const uint32_t key = rel[u][e];
-          if ((key >> hi) == pre) {
+      for (int e = 0; e < 4; ++e) {
+        const float x = v[u][e], d = x - lo_v;
+        const bool in = d >= 0.f && d <= range;
+        const uint32_t bin = __float_as_uint(fmaf(d, a, 8388610.f)) & 255u;
+        if (in && bin == (uint32_t)cut) {
+          lo_n = fminf(lo_n, x); hi_n = fmaxf(hi_n, x);
+          if (collect) {
             const int at = atomicAdd(&hcnt[288], 1);
-            if (SPADE_CHECK(at < SEL_CAND, ws.status, 305, at)) cand[at] = key;
+            if (SPADE_CHECK(at < SELR_CAND, ws.status, 305, at)) cand[at] = x;
           }
         }
       }
-      m = cnt_T;
-      __syncwarp();
     }
+    __syncwarp();
+    if (!collect) {
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) {
+        lo_n = fminf(lo_n, __shfl_xor_sync(FULL, lo_n, o));
+        hi_n = fmaxf(hi_n, __shfl_xor_sync(FULL, hi_n, o));
+      }
+      lo_v = lo_n; hi_v = hi_n;
+      continue;
+    }
+    // rank the m <= 64 values: lane l owns cand[l] and cand[32 + l]
+    const float qnan = __int_as_float(0x7fffffff);
+    const float a0 = lane < m ? cand[lane] : qnan, a1 = lane + 32 < m ? cand[lane + 32] : qnan;
+    int gt0 = 0, ge0 = 0, gt1 = 0, ge1 = 0;
+    for (int j = 0; j < m; ++j) {
+      const float b = cand[j];
+      gt0 += b > a0 ? 1 : 0; ge0 += b >= a0 ? 1 : 0;
+      gt1 += b > a1 ? 1 : 0; ge1 += b >= a1 ? 1 : 0;
+    }
+    const bool c0 = lane < m && gt0 < need_r && need_r <= ge0, c1 = lane + 32 < m && gt1 < need_r && need_r <= ge1;
+    const unsigned h0 = __ballot_sync(FULL, c0), h1 = __ballot_sync(FULL, c1);
+    if (!(h0 | h1)) { all = true; break; }       // cannot happen (1 <= need_r <= m)
+    const int src = h0 ? __ffs(h0) - 1 : __ffs(h1) - 1;
+    const float Tv = __shfl_sync(FULL, h0 ? a0 : a1, src);
+    const int gt = __shfl_sync(FULL, h0 ? gt0 : gt1, src), ge = __shfl_sync(FULL, h0 ? ge0 : ge1, src);
+    T_lo = Tv; T_hi = Tv; need_t = need_r - gt; cnt_T = ge - gt;
+    break;
   }
 
-  // ---- emit ascending ids (dynamic selection united with the static masks) ---------------------------------
-  const uint8_t* colkeep = ws.colkeep + (size_t)bh * sh.NBmax;
+  // ---- the keep bitmap, then the ascending id list ----------------------------------------------------------
   if (sh.masks_on && ws.rowfull[(size_t)bh * sh.NBmax + row]) all = true;
   uint32_t* bits = ws.rowbits + ((size_t)bh * sh.NBvmax + row) * sh.bits_ld;      // the same list as a bitmap, for k_pair_axis
-  int count = 0;
+  const int nw = (n + 31) >> 5;                  // <= NV * 4 <= 64 words
   if (all) {
-    for (int j = lane; j < n; j += 32)
-      if (SPADE_CHECK(j < sh.cap, ws.status, 302, j)) out[j] = j;
-    for (int wd = lane; wd * 32 < n; wd += 32) bits[wd] = n - wd * 32 >= 32 ? 0xffffffffu : (1u << (n - wd * 32)) - 1u;
-    count = n;
+    for (int wd = lane; wd < nw; wd += 32) words[wd] = n - wd * 32 >= 32 ? 0xffffffffu : (1u << (n - wd * 32)) - 1u;
+  } else if (need_t >= cnt_T) {
+    // every block at the cut value is kept: keep <=> v >= T_lo
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+      if (u * 128 >= n) break;
+      uint32_t kn = 0u;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) kn |= (v[u][e] >= T_lo ? 1u : 0u) << e;
+      uint32_t w = kn << (4 * (lane & 7));
+      w |= __shfl_xor_sync(FULL, w, 1);
+      w |= __shfl_xor_sync(FULL, w, 2);
+      w |= __shfl_xor_sync(FULL, w, 4);
+      if ((lane & 7) == 0) words[u * 4 + (lane >> 3)] = w;
+    }
   } else {
-    const bool ties = need < cnt_T;              // only some of the keys equal to T are kept: rank them by id
-    const int r_w = row % g.nbw, r_h = (row / g.nbw) % g.nbh, r_t = row / (g.nbw * g.nbh);
-    // The comparisons run over the registers once (straight-line code that every row executes a single time is
-    // bound by instruction fetch, so it is kept short); the keep bits of a lane's four blocks per vector are packed
-    // into one 64-bit word and the list is written by a rolled loop over the vectors.
+    // only need_t of the cnt_T blocks at the cut are kept: rank them by id
     unsigned long long knp = 0ull, eqp = 0ull;
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
       if (u * 128 >= n) break;
-      const int left = n - (u * 32 + lane) * 4;
-      uint32_t kn = 0u;
-      if (!ties) {
+      uint32_t kn = 0u, eqn = 0u;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) kn |= (e < left && rel[u][e] >= T ? 1u : 0u) << e;
-      } else {
-        uint32_t eqn = 0u;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          kn |= (e < left && rel[u][e] > T ? 1u : 0u) << e;
-          eqn |= (e < left && rel[u][e] == T ? 1u : 0u) << e;
-        }
-        eqp |= (unsigned long long)eqn << (4 * u);
+      for (int e = 0; e < 4; ++e) {
+        kn |= (v[u][e] > T_hi ? 1u : 0u) << e;
+        eqn |= (v[u][e] >= T_lo && v[u][e] <= T_hi ? 1u : 0u) << e;
       }
       knp |= (unsigned long long)kn << (4 * u);
+      eqp |= (unsigned long long)eqn << (4 * u);
     }
     int ties_seen = 0;
-    const int nvec = (n + 127) >> 7;
 #pragma unroll 1
-    for (int u = 0; u < nvec; ++u) {
-      const int j0 = (u * 32 + lane) * 4, left = n - j0;
-      uint32_t kn = (uint32_t)(knp >> (4 * u)) & 15u;      // keep bits of this lane's four blocks
-      if (ties) {
-        const uint32_t eqn = (uint32_t)(eqp >> (4 * u)) & 15u;
-        const int c = __popc(eqn);
-        int incl = c;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int up = __shfl_up_sync(FULL, incl, o);
-          if (lane >= o) incl += up;
-        }
-        int r = ties_seen + incl - c;
-#pragma unroll
-        for (int e = 0; e < 4; ++e)
-          if ((eqn >> e) & 1u) { if (r < need) kn |= 1u << e; ++r; }
-        ties_seen += __shfl_sync(FULL, incl, 31);
-      }
-      if (sh.masks_on) {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int j = j0 + e;
-          if (e < left) {
-            bool k = colkeep[j] != 0;
-            if (sh.window >= 0) {
-              const int dw = j % g.nbw - r_w, dh = (j / g.nbw) % g.nbh - r_h, dt = j / (g.nbw * g.nbh) - r_t;
-              k = k || (abs(dw) <= sh.window && abs(dh) <= sh.window && abs(dt) <= sh.window);
-            }
-            kn |= (k ? 1u : 0u) << e;
-          }
-        }
-      }
-      const int c = __popc(kn);
+    for (int u = 0; u * 128 < n; ++u) {
+      uint32_t kn = (uint32_t)(knp >> (4 * u)) & 15u;
+      const uint32_t eqn = (uint32_t)(eqp >> (4 * u)) & 15u;
+      const int c = __popc(eqn);
       int incl = c;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         const int up = __shfl_up_sync(FULL, incl, o);
         if (lane >= o) incl += up;
       }
-      int pos = count + incl - c;
+      int r = ties_seen + incl - c;
 #pragma unroll
       for (int e = 0; e < 4; ++e)
-        if ((kn >> e) & 1u) {
-          if (SPADE_CHECK(pos < sh.cap, ws.status, 303, pos)) out[pos] = j0 + e;
-          ++pos;
-        }
-      count += __shfl_sync(FULL, incl, 31);
+        if ((eqn >> e) & 1u) { if (r < need_t) kn |= 1u << e; ++r; }
+      ties_seen += __shfl_sync(FULL, incl, 31);
       uint32_t w = kn << (4 * (lane & 7));
       w |= __shfl_xor_sync(FULL, w, 1);
       w |= __shfl_xor_sync(FULL, w, 2);
       w |= __shfl_xor_sync(FULL, w, 4);
-      if ((lane & 7) == 0 && (u * 4 + (lane >> 3)) * 32 < n) bits[u * 4 + (lane >> 3)] = w;
+      if ((lane & 7) == 0) words[u * 4 + (lane >> 3)] = w;
     }
   }
+  __syncwarp();
+  // lane l owns words l and 32 + l: static masks, the bitmap row, and the ids of its set bits
+  uint32_t w0 = lane < nw ? words[lane] : 0u, w1 = lane + 32 < nw ? words[lane + 32] : 0u;
+  if (sh.masks_on && !all) {
+    const uint8_t* colkeep = ws.colkeep + (size_t)bh * sh.NBmax;
+    const int r_w = row % g.nbw, r_h = (row / g.nbw) % g.nbh, r_t = row / (g.nbw * g.nbh);
+#pragma unroll 1
+    for (int half = 0; half < 2; ++half) {
+      const int wi = lane + 32 * half;
+      if (wi >= nw) continue;
+      uint32_t add = 0u;
+      for (int bit = 0; bit < 32; ++bit) {
+        const int j = wi * 32 + bit;
+        if (j >= n) break;
+        bool k = colkeep[j] != 0;
+        if (sh.window >= 0) {
+          const int dw = j % g.nbw - r_w, dh = (j / g.nbw) % g.nbh - r_h, dt = j / (g.nbw * g.nbh) - r_t;
+          k = k || (abs(dw) <= sh.window && abs(dh) <= sh.window && abs(dt) <= sh.window);
+        }
+        add |= (k ? 1u : 0u) << bit;
+      }
+      if (half) w1 |= add; else w0 |= add;
+    }
+  }
+  if (lane < nw) bits[lane] = w0;
+  if (lane + 32 < nw) bits[lane + 32] = w1;
+  const int c0 = __popc(w0), c1 = __popc(w1);
+  int i0 = c0, i1 = c1;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int x = __shfl_up_sync(FULL, i0, o), y = __shfl_up_sync(FULL, i1, o);
+    if (lane >= o) { i0 += x; i1 += y; }
+  }
+  const int tot0 = __shfl_sync(FULL, i0, 31), tot1 = __shfl_sync(FULL, i1, 31);
+#pragma unroll 1
+  for (int half = 0; half < 2; ++half) {
+    uint32_t w = half ? w1 : w0;
+    int pos = half ? tot0 + i1 - c1 : i0 - c0;
+    const int base = (lane + 32 * half) * 32;
+    while (w) {
+      const int bit = __ffs(w) - 1;
+      w &= w - 1;
+      if (SPADE_CHECK(pos < sh.cap, ws.status, 303, pos)) out[pos] = base + bit;
+      ++pos;
+    }
+  }
+  const int count = tot0 + tot1;
   for (int j = lane; j < g.NBt; j += 32)
     if (SPADE_CHECK(count + j < sh.cap, ws.status, 306, count + j)) out[count + j] = n + j;     // text KV blocks are always kept
   if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt;
