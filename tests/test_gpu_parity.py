@@ -137,6 +137,66 @@ def test_keep_one_and_keep_all():
     _run(base.replace(mode="topp", value=1.0))
 
 
+@pytest.mark.parametrize("grid,value", [((16, 32, 32), 0.8), ((16, 32, 32), 0.45), ((20, 32, 64), 0.8)])
+def test_topk_rows_with_ties_and_clusters_are_the_exact_top_k_lowest_ids_first(grid, value):
+    """Score rows that hold large groups of equal or nearly equal values (more than the 64 the index search ranks
+    directly, so its histogram is refined between the group's own extremes, and rows where every score is the
+    same): the list must agree with the oracle away from the cut, and be the exact top-k of the fp32 table the
+    search read: nothing dropped scores higher than something kept, equal scores go by lower id."""
+    from tests import parity_util as pu
+    from oracle import spade_oracle as so
+    from paper_2608_03335_b200.workloads import make_qkv, bf16_bits
+    w = small_variant(WORKLOADS["wan14b"], heads=3, grid=grid).replace(mode="sparsity", value=value)
+    blk = w.candidates[0]
+    g = so.geometry(w.grid, w.n_text, blk)
+    nbv = g["NBv"]
+    assert nbv >= 256 and all(x % b == 0 for x, b in zip(grid, blk))
+    Q, K, V = make_qkv(w, "cuda")
+    K = K.clone()
+    tok = [torch.as_tensor(so.block_tokens(w.grid, w.n_text, blk, b), device="cuda", dtype=torch.long) for b in range(nbv)]
+    c0 = K[0, 0, tok[3][0]].clone()                    # head 0: blocks 0..99 made of one token value -> 100 equal scores per row
+    for b in range(100):
+        K[0, 0, tok[b]] = c0
+    c1 = K[0, 1, tok[7][5]].clone()                    # head 1: every key the same -> every row one value
+    K[0, 1, :, :] = c1
+    c2 = K[0, 2, tok[11][1]].clone()                   # head 2: blocks 50..179 one value each, a bf16 step or two apart
+    for b in range(50, 180):
+        K[0, 2, tok[b]] = c2
+        ch = (b * 5) % w.d
+        step = c2[ch].abs().float() * 2.0 ** -7 + 2.0 ** -20
+        K[0, 2, tok[b][: 1 + b // 64], ch] = (c2[ch].float() + step).to(torch.bfloat16)
+    K = K.contiguous()
+    BH = w.batch * w.heads
+    qb, kb = (bf16_bits(x).reshape(BH, w.n_tokens, w.d) for x in (Q, K))
+    plan = pu.make_plan(w)
+    try:
+        forced = [0, 0, 0]
+        plan.spade_plan(Q, K, forced_scheme=forced)
+        plan.spade_summarize(Q, K)
+        plan.spade_select()
+        plan.spade_status()
+        torch.cuda.synchronize()
+        rep = pu.Report()
+        pu.check_select(w, plan, qb, kb, forced, rep)
+        t = plan.tables()
+        keep = t["keep"].cpu().numpy()
+        kv_idx, kv_cnt = t["kv_idx"].cpu().numpy(), t["kv_cnt"].cpu().numpy()
+        big_groups = 0
+        for bh in range(BH):
+            S = t["block_scores"][bh, :nbv, :nbv].cpu().numpy()
+            k = int(keep[bh])
+            for i in range(nbv):
+                kept = kv_idx[bh, i, :kv_cnt[bh, i]].tolist()
+                order = sorted(range(nbv), key=lambda j: (-S[i, j], j))
+                assert kept == sorted(order[:k]), f"head {bh} row {i}: not the top {k} by (score, lower id)"
+                cut = S[i, order[k - 1]]
+                big_groups += int((np.abs(S[i] - cut) <= 1e-3 * max(abs(cut), 1e-6)).sum() > 64)
+        assert big_groups > nbv, "the inputs did not put large groups at the cut"
+        print(f"[ties {grid} {value}] rows {rep.rows_checked} near-cut {rep.near_cut_blocks}, rows with > 64 values at the cut: {big_groups}")
+    finally:
+        plan.close()
+
+
 def test_caller_written_lists_and_empty_rows():
     """spade_attn on lists the caller wrote: random masks, and an empty row gives zeros."""
     from oracle import spade_oracle as so
