@@ -515,10 +515,11 @@ int spade_summarize(spade_plan_t* p, const void* Q, const void* K, void* ws, voi
   if ((rc = check_tensor(Q, "Q")) || (rc = check_tensor(K, "K"))) return rc;
   if (p->stage < 1 || p->stage_ws != ws) return fail(SPADE_ERR_ORDER, "spade_summarize needs spade_plan on this workspace first");
   ON_PLAN_DEVICE(p);
-  if (p->have_csum) CUDA_TRY(launch_gather(p->sh, p->gp, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
+  // the copy of the chosen candidate's sums also writes the estimator's split K'; the token pass needs a kernel for it
+  if (p->have_csum) CUDA_TRY(launch_gather(p->sh, p->gp, tables_at(p, ws), p->num_sms, p->sh.estimator == 0, (cudaStream_t)stream));
   else CUDA_TRY(launch_summarize(Q, K, p->sh, p->gp, p->st, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
   p->launches += 1;
-  if (!p->sh.estimator) {
+  if (!p->sh.estimator && !p->have_csum) {
     CUDA_TRY(launch_split_k(p->sh, p->gp, tables_at(p, ws), p->num_sms, (cudaStream_t)stream));
     p->launches += 1;
   }

@@ -362,18 +362,19 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
 
 // SICS(block) = |sum_t q_t / |q_t||^2 (Eq. 4 / Algorithm 1) from the summed unit vectors the one-pass kernel left:
 // one warp per (head, tensor, candidate, video block), channels in a fixed order.
+template <class Index>      // int when the number of blocks fits (64-bit division costs a call per block), long otherwise
 __global__ void __launch_bounds__(256)
 k_sics_from_sums(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, const WsTables ws) {
   const int lane = threadIdx.x & 31;
-  const long gw = (long)blockIdx.x * 8 + (threadIdx.x >> 5), nw = (long)gridDim.x * 8;
-  const long total = (long)sh.BH * 2 * sh.units_per_ht;
-  for (long u0 = gw * 4; u0 < total; u0 += nw * 4) {           // four blocks per warp and step: four loads in flight
+  const Index gw = (Index)blockIdx.x * 8 + (threadIdx.x >> 5), nw = (Index)gridDim.x * 8;
+  const Index total = (Index)sh.BH * 2 * sh.units_per_ht;
+  for (Index u0 = gw * 4; u0 < total; u0 += nw * 4) {           // four blocks per warp and step: four loads in flight
     float4 v[4];
     size_t out[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const long u = u0 + q < total ? u0 + q : total - 1;
-      const int ht = (int)(u / sh.units_per_ht), rem = (int)(u % sh.units_per_ht);
+      const Index u = u0 + q < total ? u0 + q : total - 1;
+      const int ht = (int)(u / (Index)sh.units_per_ht), rem = (int)(u % (Index)sh.units_per_ht);
       int c = 0;
 #pragma unroll
       for (int i = 1; i < SPADE_MAX_CANDS; ++i)
@@ -528,6 +529,7 @@ cudaError_t launch_plan_fused(const PlanMaps* maps, const void* Q, const void* K
   const long blocks = (long)sh.BH * 2 * sh.units_per_ht;
   long ctas = (blocks + 31) / 32;
   if (ctas > (long)num_sms * 8) ctas = (long)num_sms * 8;
-  k_sics_from_sums<<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
+  if (blocks + 4l * num_sms * 64 < 0x7fffffffl) k_sics_from_sums<int><<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
+  else k_sics_from_sums<long><<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
   return cudaGetLastError();
 }

@@ -244,7 +244,7 @@ k_static(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
 
 // Summaries of the chosen scheme, picked out of the all-candidate table of the block pass.
 __global__ void __launch_bounds__(256)
-k_gather(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws) {
+k_gather(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws, const int split) {
   const long total = (long)sh.BH * 2 * sh.NBmax * 32;       // float4 elements
   for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
     const int c4 = (int)(i & 31);
@@ -252,9 +252,22 @@ k_gather(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, W
     const int b = (int)(rowi % sh.NBmax), ht = (int)(rowi / sh.NBmax);
     const int bh = ht >> 1, tensor = ht & 1;
     const int c = ws.scheme[bh];
-    if (b >= gp.g[c].NB) continue;
-    const float4 v = reinterpret_cast<const float4*>(ws.csum + ((((size_t)ht * sh.C + c) * sh.NBmax) + b) * SPADE_D)[c4];
-    reinterpret_cast<float4*>((tensor ? ws.ksum : ws.qsum) + ((size_t)bh * sh.NBmax + b) * SPADE_D)[c4] = v;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (b < gp.g[c].NB) {
+      v = reinterpret_cast<const float4*>(ws.csum + ((((size_t)ht * sh.C + c) * sh.NBmax) + b) * SPADE_D)[c4];
+      reinterpret_cast<float4*>((tensor ? ws.ksum : ws.qsum) + ((size_t)bh * sh.NBmax + b) * SPADE_D)[c4] = v;
+    }
+    if (split && tensor) {
+      // the estimator's operand B as k_split_k writes it: K' of the video blocks as TF32 value and remainder, zero rows behind them
+      if (b >= gp.g[c].NBv) v = make_float4(0.f, 0.f, 0.f, 0.f);
+      float4 h, l;
+      h.x = __uint_as_float((__float_as_uint(v.x) + 0x1000u) & 0xffffe000u); l.x = v.x - h.x;
+      h.y = __uint_as_float((__float_as_uint(v.y) + 0x1000u) & 0xffffe000u); l.y = v.y - h.y;
+      h.z = __uint_as_float((__float_as_uint(v.z) + 0x1000u) & 0xffffe000u); l.z = v.z - h.z;
+      h.w = __uint_as_float((__float_as_uint(v.w) + 0x1000u) & 0xffffe000u); l.w = v.w - h.w;
+      reinterpret_cast<float4*>(ws.ksplit + (((size_t)bh * 2 + 0) * sh.NBmax + b) * SPADE_D)[c4] = h;
+      reinterpret_cast<float4*>(ws.ksplit + (((size_t)bh * 2 + 1) * sh.NBmax + b) * SPADE_D)[c4] = l;
+    }
   }
 }
 
@@ -1284,11 +1297,11 @@ cudaError_t launch_static(const Shape& sh, const GeoPack& gp, const StaticTables
   return cudaGetLastError();
 }
 
-cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s) {
+cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, int split, cudaStream_t s) {
   const long total = (long)sh.BH * 2 * sh.NBmax * 32;
   long ctas = (total + 255) / 256;
   if (ctas > (long)num_sms * 16) ctas = (long)num_sms * 16;
-  k_gather<<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws);
+  k_gather<<<(unsigned)ctas, 256, 0, s>>>(sh, gp, ws, split);
   return cudaGetLastError();
 }
 

@@ -154,7 +154,7 @@ cudaError_t launch_cells(const void* Q, const void* K, const Shape& sh, const Ws
 cudaError_t launch_blocks(const void* Q, const void* K, const Shape& sh, const GeoPack& gp, const StaticTables& st,
                           const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_static(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws, cudaStream_t s);
-cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
+cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, int split, cudaStream_t s);
 cudaError_t launch_split_k(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_choose(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
                           const ForcedPack& forced, int have_sics, cudaStream_t s);
