@@ -1012,12 +1012,12 @@ k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
 // are consecutive ids: eight lanes' nibbles make a word of the row's bitmap, and the ascending id list is written
 // from the bitmap words.
 constexpr int SELR_CAND = 64;
-constexpr int SELR_WORDS = 296 + SELR_CAND + 64;   // per warp: 256 bin counts, 32 dump slots, list counter (word 288); candidates; bitmap words
+constexpr int SELR_WORDS = 296 + SELR_CAND + 8 + 64;   // per warp: 256 bin counts, 32 dump slots, list counter (word 288); candidates (+ 8 of padding); bitmap words
 
 template <int NV>
 __global__ void __launch_bounds__(SEL_R * 32, 3)
 k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws) {
-  __shared__ int sel_sm[SEL_R * SELR_WORDS];
+  __shared__ __align__(16) int sel_sm[SEL_R * SELR_WORDS];
   const int bh = blockIdx.y;
   const CandGeo& g = gp.g[ws.scheme[bh]];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1033,7 +1033,7 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
   }
   int* hcnt = sel_sm + warp * SELR_WORDS;                        // [256] bins, [256 + lane] dump slots, [288] list counter
   float* cand = reinterpret_cast<float*>(hcnt + 296);            // [SELR_CAND]
-  uint32_t* words = reinterpret_cast<uint32_t*>(hcnt + 296 + SELR_CAND);     // [64] the row's keep bitmap
+  uint32_t* words = reinterpret_cast<uint32_t*>(hcnt + 296 + SELR_CAND + 8);     // [64] the row's keep bitmap
   const int ldc = sh.ld_scores;
 
   // ---- the row: NV float4 per lane; slots past the row's end hold NaN, which fails every comparison below ----------
@@ -1127,11 +1127,18 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
     // rank the m <= 64 values: lane l owns cand[l] and cand[32 + l]
     const float qnan = __int_as_float(0x7fffffff);
     const float a0 = lane < m ? cand[lane] : qnan, a1 = lane + 32 < m ? cand[lane + 32] : qnan;
+    __syncwarp();
+    if (lane < 8) cand[m + lane] = qnan;          // the loop below reads eight at a time; NaN counts for nothing
+    __syncwarp();
     int gt0 = 0, ge0 = 0, gt1 = 0, ge1 = 0;
-    for (int j = 0; j < m; ++j) {
-      const float b = cand[j];
-      gt0 += b > a0 ? 1 : 0; ge0 += b >= a0 ? 1 : 0;
-      gt1 += b > a1 ? 1 : 0; ge1 += b >= a1 ? 1 : 0;
+    for (int j0 = 0; j0 < m; j0 += 8) {
+      const float4 ba = *reinterpret_cast<const float4*>(cand + j0), bb = *reinterpret_cast<const float4*>(cand + j0 + 4);
+      const float b[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        gt0 += b[k] > a0 ? 1 : 0; ge0 += b[k] >= a0 ? 1 : 0;
+        gt1 += b[k] > a1 ? 1 : 0; ge1 += b[k] >= a1 ? 1 : 0;
+      }
     }
     const bool c0 = lane < m && gt0 < need_r && need_r <= ge0, c1 = lane + 32 < m && gt1 < need_r && need_r <= ge1;
     const unsigned h0 = __ballot_sync(FULL, c0), h1 = __ballot_sync(FULL, c1);
