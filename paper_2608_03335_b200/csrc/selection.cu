@@ -4,7 +4,7 @@
 //   k_groups     heads ordered by chosen scheme + attention work-item prefix (Sec. 3.3, head grouping)
 //   k_summarize  mean summaries Q', K' of the chosen scheme (Sec. 3.1 Summarizer Expression)
 //   k_minmax     channel-wise max / min summaries; k_scores_minmax: the estimators built on them (Fig. 4a, 4b)
-//   k_select     index search on the block scores: softmax over KV blocks, Top-K / Top-P, ascending lists
+//   k_select_reg index search on the block scores: softmax over KV blocks, Top-K / Top-P, ascending lists
 //                (the scores S = <Q'_i,K'_j>/sqrt(d) come from k_scores in scores.cu)
 #include "spade_common.cuh"
 
@@ -741,23 +741,11 @@ k_scores_minmax(const __grid_constant__ Shape sh, const __grid_constant__ GeoPac
 // ------------------------------------------------------------------------------------------------
 // Estimator + index search.
 constexpr int SEL_R = 8;        // query-block rows per CTA; one warp per row
-constexpr int SEL_CAND = 256;   // keys of the bin the cut falls in that the later radix passes work on
-constexpr int SEL_WARP_WORDS = 256 + 512 + SEL_CAND;   // per warp: bin counts, 64-bit bin masses, candidate keys
-
-__device__ __forceinline__ uint32_t order_key(float s) {      // larger float <=> larger key
-  const uint32_t u = __float_as_uint(s);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float key_to_float(uint32_t k) {
-  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-}
-
 // Scan a 256-bin histogram from the top bin down; find the first NON-EMPTY bin at which
 // `above + cumulative >= need`.  Lane l owns bins 255-8l .. 248-8l.  Returns the bin (or -1 when the
 // total never reaches `need`) and adds the weight of the bins above it to `above`.  All lanes get the
-// same result.  With floating-point weights the lane-level scan and the in-lane running sum round
-// differently, so the crossing is only ever placed in a bin that holds something: an empty bin would
-// leave the next pass of the descent without a single matching key.
+// same result.  The crossing is only ever placed in a bin that holds something: an empty bin would
+// leave the next pass without a single value.
 template <class T>
 __device__ __forceinline__ int find_bin(const T* hist, T need, T& above, int lane) {
   T v[8], tot = 0;
@@ -796,228 +784,28 @@ __device__ __forceinline__ int find_bin(const T* hist, T need, T& above, int lan
   return bin;
 }
 
-// Index search: one warp per query block reads its row of block scores (written by k_scores) into
-// shared memory and picks the kept KV blocks.
-__global__ void __launch_bounds__(SEL_R * 32, 2)
-k_select(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws) {
-  extern __shared__ __align__(16) float smem[];
-  const int bh = blockIdx.y;
-  const CandGeo& g = gp.g[ws.scheme[bh]];
-  const int row0 = blockIdx.x * SEL_R;
-  if (row0 >= g.NB) return;
-  const int n = g.NBv;                         // video KV blocks compete; text blocks are appended
-  const int ldc = sh.ld_scores;
-  float* sc = smem;                            // [SEL_R][ldc]
-  float* sk = sc + SEL_R * ldc;                // per-warp histograms
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (row0 + warp < n) {
-    const float4* src = reinterpret_cast<const float4*>(ws.scores + ((size_t)bh * sh.NBvmax + row0 + warp) * ldc);
-    float4* dst = reinterpret_cast<float4*>(sc + warp * ldc);
-    const int n4 = (n + 3) / 4;
-    for (int i0 = 0; i0 < n4; i0 += 256) {            // eight 16-byte loads in flight per lane
-      float4 v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int i = i0 + u * 32 + lane;
-        if (i < n4) v[u] = __ldcs(src + i);
-      }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int i = i0 + u * 32 + lane;
-        if (i < n4) dst[i] = v[u];
-      }
-    }
-  }
-  __syncwarp();
-
-  // ---- phase 2: one warp per query block ---------------------------------------------------------
-  const int row = row0 + warp;
-  if (row >= g.NB) return;
-  int* out = ws.kv_idx + ((size_t)bh * sh.NBmax + row) * sh.cap;
-  int count = 0;
-  if (row >= n) {                               // text query block: every block
-    for (int j = lane; j < g.NB; j += 32)
-      if (SPADE_CHECK(j < sh.cap, ws.status, 301, j)) out[j] = j;
-    if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = g.NB;
-    return;
-  }
-  const float* s = sc + warp * ldc;
-  int* hcnt = reinterpret_cast<int*>(sk) + warp * (sh.mode == 1 ? SEL_WARP_WORDS : SEL_WARP_WORDS - 512);   // [256] counts per radix bin
-  unsigned long long* hmass = reinterpret_cast<unsigned long long*>(hcnt + 256);     // [256] softmax mass per bin, fixed point
-  uint32_t* cand = reinterpret_cast<uint32_t*>(hcnt + (sh.mode == 1 ? 768 : 256));   // [SEL_CAND] rel keys still in the race (over the unused masses in Top-K mode)
-  const unsigned lt = (1u << lane) - 1u;
-
-  // Keys replace the scores in place; the radix descent starts below the bits every key of the row
-  // shares (sign and most of the exponent), so each 8-bit pass spreads over many bins.
-  uint32_t* ks = reinterpret_cast<uint32_t*>(sc + warp * ldc);
-  uint32_t kmax = 0u, kmin = 0xffffffffu;
-  for (int j = lane; j < n; j += 32) {
-    const uint32_t key = order_key(s[j]);
-    ks[j] = key;
-    kmax = max(kmax, key);
-    kmin = min(kmin, key);
-  }
-#pragma unroll
-  for (int o = 16; o >= 1; o >>= 1) {
-    kmax = max(kmax, __shfl_xor_sync(FULL, kmax, o));
-    kmin = min(kmin, __shfl_xor_sync(FULL, kmin, o));
-  }
-  __syncwarp();
-  // The descent works on rel = key - kmin, whose top bits spread over the row's actual range of values
-  // (a common bit prefix would not: rows that straddle zero differ in the sign bit already).
-  int hi = kmax != kmin ? 32 - __clz(kmax - kmin) : 0;         // rel < 2^hi
-  uint32_t T = 0u;                                              // becomes rel of the last kept value
-  int need = 0;         // how many blocks with key == T are kept (lowest ids first)
-  bool all = false;
-  // The first pass of the descent scans the whole row.  As soon as the bin the cut falls in holds at most
-  // SEL_CAND keys they are copied out, and the remaining passes (down to bit 0) only touch that short list.
-  int m = -1;           // -1: the candidates are the whole row; >= 0: cand[0 .. m)
-  auto compact = [&](int cnt) {
-    if (m >= 0 || hi == 0 || cnt > SEL_CAND) return;
-    int at = 0;
-    for (int j0 = 0; j0 < n; j0 += 32) {
-      const int j = j0 + lane;
-      const uint32_t key = j < n ? ks[j] - kmin : 0u;
-      const bool hit = j < n && (key >> hi) == (T >> hi);
-      const unsigned bm = __ballot_sync(FULL, hit);
-      if (hit && SPADE_CHECK(at + __popc(bm & lt) < SEL_CAND, ws.status, 305, at)) cand[at + __popc(bm & lt)] = key;
-      at += __popc(bm);
-    }
-    m = at;
-    __syncwarp();
-  };
-  if (sh.mode != 1) {
-    // Top-K: radix select of the k-th largest key, up to 8 bits per pass.
-    need = ws.keep[bh];
-    if (need >= n) all = true;
-    while (hi > 0 && !all) {
-      const int lo = hi > 8 ? hi - 8 : 0;
-      const uint32_t bmask = (1u << (hi - lo)) - 1u;
-      for (int i = lane; i < 256; i += 32) hcnt[i] = 0;
-      __syncwarp();
-      const int cnt_all = m < 0 ? n : m;
-      const uint32_t* src = m < 0 ? ks : cand;
-      const uint32_t base = m < 0 ? kmin : 0u;                     // the candidate list holds rel already
-      for (int j = lane; j < cnt_all; j += 32) {
-        const uint32_t key = src[j] - base;
-        if ((hi >= 32 || (key >> hi) == (T >> hi)) && SPADE_CHECK(((key >> lo) & bmask) < 256u, ws.status, 304, (key >> lo) & bmask))
-          atomicAdd(&hcnt[(key >> lo) & bmask], 1);
-      }
-      __syncwarp();
-      int above = 0;
-      const int bin = find_bin<int>(hcnt, need, above, lane);
-      if (bin < 0) { all = true; break; }          // cannot happen (need <= keys under the prefix); keep the row whole if it does
-      T |= (uint32_t)bin << lo;
-      need -= above;
-      hi = lo;
-      const int cnt = hcnt[bin];
-      __syncwarp();
-      compact(cnt);
-    }
-  } else {
-    // Top-P: the same descent on softmax mass.  Weights exp(s - max) are summed in 2^-40 fixed point:
-    // integer sums do not depend on the order the lanes add them in, so the lists are reproducible bit for
-    // bit, and the mass of a bin equals the sum of its sub-bins in the next pass exactly.
-    const float mx = key_to_float(kmax);
-    auto weight = [&](uint32_t rel) -> unsigned long long {
-      return __float2ull_rn(expf(key_to_float(rel + kmin) - mx) * 1099511627776.f);
-    };
-    unsigned long long z = 0ull;
-    for (int j = lane; j < n; j += 32) z += weight(ks[j] - kmin);
-#pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) z += __shfl_xor_sync(FULL, z, o);
-    unsigned long long target = (unsigned long long)ceil((double)ws.pthr[bh] * (double)z);
-    if (target > z) target = z;
-    if (target == 0ull) target = 1ull;
-    unsigned long long above = 0ull;
-    int cnt_T = n;
-    while (hi > 0 && !all) {
-      const int lo = hi > 8 ? hi - 8 : 0;
-      const uint32_t bmask = (1u << (hi - lo)) - 1u;
-      for (int i = lane; i < 256; i += 32) { hcnt[i] = 0; hmass[i] = 0ull; }
-      __syncwarp();
-      const int cnt_all = m < 0 ? n : m;
-      const uint32_t* src = m < 0 ? ks : cand;
-      const uint32_t base = m < 0 ? kmin : 0u;
-      for (int j = lane; j < cnt_all; j += 32) {
-        const uint32_t key = src[j] - base;
-        if (hi >= 32 || (key >> hi) == (T >> hi)) {
-          atomicAdd(&hcnt[(key >> lo) & bmask], 1);
-          atomicAdd(&hmass[(key >> lo) & bmask], weight(key));
-        }
-      }
-      __syncwarp();
-      const int bin = find_bin<unsigned long long>(hmass, target, above, lane);
-      if (bin < 0) { all = true; break; }            // cannot happen (target <= total mass under the prefix)
-      T |= (uint32_t)bin << lo;
-      cnt_T = hcnt[bin];
-      hi = lo;
-      __syncwarp();
-      compact(cnt_T);
-    }
-    if (!all) {
-      // every key equal to T carries the same weight: how many of them (lowest ids first) the mass still needs
-      const unsigned long long wT = weight(T);
-      unsigned long long t = wT > 0ull ? (target - above + wT - 1ull) / wT : (unsigned long long)cnt_T;
-      if (target <= above) t = 1ull;
-      need = (int)(t < 1ull ? 1ull : (t > (unsigned long long)cnt_T ? (unsigned long long)cnt_T : t));
-    }
-  }
-
-  // ---- emit ascending ids (dynamic selection united with the static masks) ---------------------------
-  const uint8_t* colkeep = ws.colkeep + (size_t)bh * sh.NBmax;
-  if (sh.masks_on && ws.rowfull[(size_t)bh * sh.NBmax + row]) all = true;
-  const int r_w = row % g.nbw, r_h = (row / g.nbw) % g.nbh, r_t = row / (g.nbw * g.nbh);
-  uint32_t* bits = ws.rowbits + ((size_t)bh * sh.NBvmax + row) * sh.bits_ld;      // the same list as a bitmap, for k_pair_axis
-  if (all) {
-    for (int j = lane; j < n; j += 32)
-      if (SPADE_CHECK(j < sh.cap, ws.status, 302, j)) out[j] = j;
-    for (int wd = lane; wd * 32 < n; wd += 32) bits[wd] = n - wd * 32 >= 32 ? 0xffffffffu : (1u << (n - wd * 32)) - 1u;
-    count = n;
-  } else {
-    int ties_seen = 0;
-    for (int j0 = 0; j0 < n; j0 += 32) {
-      const int j = j0 + lane;
-      const bool in = j < n;
-      const uint32_t key = in ? ks[j] - kmin : 0u;
-      const bool eq = in && key == T, gt = in && key > T;
-      const unsigned em = __ballot_sync(FULL, eq);
-      bool keep = gt || (eq && ties_seen + __popc(em & lt) < need);
-      if (sh.masks_on && in) {
-        keep = keep || colkeep[j] != 0;
-        if (sh.window >= 0) {
-          const int dw = j % g.nbw - r_w, dh = (j / g.nbw) % g.nbh - r_h, dt = j / (g.nbw * g.nbh) - r_t;
-          keep = keep || (abs(dw) <= sh.window && abs(dh) <= sh.window && abs(dt) <= sh.window);
-        }
-      }
-      const unsigned km = __ballot_sync(FULL, keep);
-      if (lane == 0) bits[j0 >> 5] = km;
-      if (keep && SPADE_CHECK(count + __popc(km & lt) < sh.cap, ws.status, 303, count)) out[count + __popc(km & lt)] = j;
-      count += __popc(km);
-      ties_seen += __popc(em);
-    }
-  }
-  for (int j = lane; j < g.NBt; j += 32)
-    if (SPADE_CHECK(count + j < sh.cap, ws.status, 306, count + j)) out[count + j] = n + j;     // text KV blocks are always kept
-  if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt;
-}
-
-// Top-K index search with the row held in registers (rows of up to NV * 128 blocks).  The scores are read once
+// Index search (Sec. 3.1, 3.3) with the row held in registers (rows of up to NV * 128 blocks; a plan takes at most 2048).  The scores are read once
 // into NV float4 per lane.  The k-th largest value is found by histogram passes that are LINEAR in the value
 // between the smallest and largest score still in the race (250 bins), so that a row of roughly bell-shaped
 // scores leaves a dozen values in the bin the cut falls in; up to 64 of them are then ranked directly (every
 // lane counts how many are larger than its own).  A bin with more than 64 is split again between its own
 // minimum and maximum.  Binning only decides which values are ranked: the kept set is the exact top-k of the
-// fp32 scores, ties by lower id.  Lane l holds blocks 128 u + 4 l .. + 3 of vector u, so a lane's four keep bits
+// fp32 scores, ties by lower id; text KV blocks are appended, text query rows list every block.  Lane l holds blocks 128 u + 4 l .. + 3 of vector u, so a lane's four keep bits
 // are consecutive ids: eight lanes' nibbles make a word of the row's bitmap, and the ascending id list is written
 // from the bitmap words.
+//
+// Top-P (TOPP) runs the same passes on softmax mass: exp(s - max) in 2^-40 fixed point (integer sums do not
+// depend on the order the lanes add them in, and a bin's mass equals the sum of its values' masses exactly); the ranking
+// loop then also adds up the mass of the values above each candidate.
 constexpr int SELR_CAND = 64;
 constexpr int SELR_WORDS = 296 + SELR_CAND + 8 + 64;   // per warp: 256 bin counts, 32 dump slots, list counter (word 288); candidates (+ 8 of padding); bitmap words
+constexpr int SELR_WORDS_P = SELR_WORDS + 512 + 2 * (SELR_CAND + 8);     // Top-P: + 256 bin masses and the candidates' masses (64-bit)
 
-template <int NV>
-__global__ void __launch_bounds__(SEL_R * 32, 3)
-k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws) {
-  __shared__ __align__(16) int sel_sm[SEL_R * SELR_WORDS];
+template <int NV, bool TOPP>
+__global__ void __launch_bounds__(SEL_R * 32, TOPP ? 2 : 3)
+k_select_reg(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws) {
+  constexpr int WORDS = TOPP ? SELR_WORDS_P : SELR_WORDS;
+  __shared__ __align__(16) int sel_sm[SEL_R * WORDS];
   const int bh = blockIdx.y;
   const CandGeo& g = gp.g[ws.scheme[bh]];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1031,9 +819,11 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
     if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = g.NB;
     return;
   }
-  int* hcnt = sel_sm + warp * SELR_WORDS;                        // [256] bins, [256 + lane] dump slots, [288] list counter
-  float* cand = reinterpret_cast<float*>(hcnt + 296);            // [SELR_CAND]
+  int* hcnt = sel_sm + warp * WORDS;                             // [256] bins, [256 + lane] dump slots, [288] list counter
+  float* cand = reinterpret_cast<float*>(hcnt + 296);            // [SELR_CAND + 8]
   uint32_t* words = reinterpret_cast<uint32_t*>(hcnt + 296 + SELR_CAND + 8);     // [64] the row's keep bitmap
+  unsigned long long* hmass = reinterpret_cast<unsigned long long*>(hcnt + SELR_WORDS);      // Top-P: [256] mass per bin
+  unsigned long long* cand_w = hmass + 256;                                                   // Top-P: [SELR_CAND + 8]
   const int ldc = sh.ld_scores;
 
   // ---- the row: NV float4 per lane; slots past the row's end hold NaN, which fails every comparison below ----------
@@ -1060,19 +850,48 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
   }
 
   // ---- the cut: keep v > T_hi, and need_t of the cnt_T blocks with T_lo <= v <= T_hi (lowest ids first) ---------------
-  int need_r = ws.keep[bh];                                       // blocks still to keep among those in [lo_v, hi_v]
-  bool all = need_r >= n;
+  int need_r = TOPP ? 1 : ws.keep[bh];                            // Top-K: blocks still to keep among those in [lo_v, hi_v]
+  bool all = !TOPP && need_r >= n;
   int m = n;                                                      // blocks in [lo_v, hi_v]
   float T_lo = 0.f, T_hi = 0.f;
   int need_t = 0, cnt_T = 0;
+  // Top-P: mass still to cover is target - above, both in 2^-40 fixed point of exp(s - max)
+  const float mx = hi_v;
+  auto weight = [&](float x) -> unsigned long long { return __float2ull_rn(expf(x - mx) * 1099511627776.f); };
+  unsigned long long target = 0ull, above_m = 0ull;
+  auto ties_for_mass = [&](unsigned long long above_T, unsigned long long wT, int cnt) -> int {
+    // every block at the cut value carries the same mass: how many of them (lowest ids first) the target still needs
+    unsigned long long t = wT > 0ull ? (target - above_T + wT - 1ull) / wT : (unsigned long long)cnt;
+    if (target <= above_T) t = 1ull;
+    return (int)(t < 1ull ? 1ull : (t > (unsigned long long)cnt ? (unsigned long long)cnt : t));
+  };
+  if constexpr (TOPP) {
+    unsigned long long z = 0ull;
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+      if (u * 128 >= n) break;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (v[u][e] >= lo_v) z += weight(v[u][e]);                // NaN (past the row's end) fails the test
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) z += __shfl_xor_sync(FULL, z, o);
+    target = (unsigned long long)ceil((double)ws.pthr[bh] * (double)z);
+    if (target > z) target = z;
+    if (target == 0ull) target = 1ull;
+  }
   for (int level = 0; !all; ++level) {
     const float range = hi_v - lo_v;
     if (!(range > 1e-30f) || level >= 40) {                       // one value left (or values no fp32 arithmetic tells apart): ties
-      T_lo = lo_v; T_hi = hi_v; need_t = need_r; cnt_T = m;
+      T_lo = lo_v; T_hi = hi_v; cnt_T = m;
+      need_t = TOPP ? ties_for_mass(above_m, weight(hi_v), m) : need_r;
       break;
     }
     const float a = 250.f / range;
-    for (int i = lane; i < 256; i += 32) hcnt[i] = 0;
+    for (int i = lane; i < 256; i += 32) {
+      hcnt[i] = 0;
+      if constexpr (TOPP) hmass[i] = 0ull;
+    }
     __syncwarp();
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
@@ -1082,14 +901,23 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
         const float d = v[u][e] - lo_v;
         const bool in = d >= 0.f && d <= range;
         const uint32_t bin = __float_as_uint(fmaf(d, a, 8388610.f)) & 255u;        // 2 .. 252, monotone in the value
-        atomicAdd(&hcnt[in ? bin : 256u + lane], 1);                             // misses go to the lane's own dump slot
+        if constexpr (TOPP) {
+          if (in) { atomicAdd(&hcnt[bin], 1); atomicAdd(&hmass[bin], weight(v[u][e])); }
+        } else {
+          atomicAdd(&hcnt[in ? bin : 256u + lane], 1);                           // misses go to the lane's own dump slot
+        }
       }
     }
     __syncwarp();
-    int above = 0;
-    const int cut = find_bin<int>(hcnt, need_r, above, lane);
-    if (cut < 0) { all = true; break; }          // cannot happen (need_r <= blocks in range); keep the row whole if it does
-    need_r -= above;
+    int cut;
+    if constexpr (TOPP) {
+      cut = find_bin<unsigned long long>(hmass, target, above_m, lane);
+    } else {
+      int above = 0;
+      cut = find_bin<int>(hcnt, need_r, above, lane);
+      need_r -= above;
+    }
+    if (cut < 0) { all = true; break; }          // cannot happen (the target is within what the range holds); keep the row whole if it does
     m = hcnt[cut];
     __syncwarp();
     // one more pass over the registers: the cut bin's own range, and (when it is short) its values
@@ -1109,7 +937,10 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
           lo_n = fminf(lo_n, x); hi_n = fmaxf(hi_n, x);
           if (collect) {
             const int at = atomicAdd(&hcnt[288], 1);
-            if (SPADE_CHECK(at < SELR_CAND, ws.status, 305, at)) cand[at] = x;
+            if (SPADE_CHECK(at < SELR_CAND, ws.status, 305, at)) {
+              cand[at] = x;
+              if constexpr (TOPP) cand_w[at] = weight(x);
+            }
           }
         }
       }
@@ -1129,6 +960,10 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
     const float a0 = lane < m ? cand[lane] : qnan, a1 = lane + 32 < m ? cand[lane + 32] : qnan;
     __syncwarp();
     if (lane < 8) cand[m + lane] = qnan;          // the loop below reads eight at a time; NaN counts for nothing
+    unsigned long long wa0 = 0ull, wa1 = 0ull, G0 = 0ull, G1 = 0ull;       // Top-P: own mass, mass of the values above
+    if constexpr (TOPP) {
+      wa0 = lane < m ? cand_w[lane] : 0ull; wa1 = lane + 32 < m ? cand_w[lane + 32] : 0ull;
+    }
     __syncwarp();
     int gt0 = 0, ge0 = 0, gt1 = 0, ge1 = 0;
     for (int j0 = 0; j0 < m; j0 += 8) {
@@ -1138,15 +973,33 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
       for (int k = 0; k < 8; ++k) {
         gt0 += b[k] > a0 ? 1 : 0; ge0 += b[k] >= a0 ? 1 : 0;
         gt1 += b[k] > a1 ? 1 : 0; ge1 += b[k] >= a1 ? 1 : 0;
+        if constexpr (TOPP) {
+          const unsigned long long wb = cand_w[j0 + k];          // past the end: unused, the comparison with NaN fails
+          G0 += b[k] > a0 ? wb : 0ull; G1 += b[k] > a1 ? wb : 0ull;
+        }
       }
     }
-    const bool c0 = lane < m && gt0 < need_r && need_r <= ge0, c1 = lane + 32 < m && gt1 < need_r && need_r <= ge1;
+    bool c0, c1;
+    if constexpr (TOPP) {
+      const unsigned long long lo0 = above_m + G0, lo1 = above_m + G1;
+      c0 = lane < m && lo0 < target && target <= lo0 + (unsigned long long)(ge0 - gt0) * wa0;
+      c1 = lane + 32 < m && lo1 < target && target <= lo1 + (unsigned long long)(ge1 - gt1) * wa1;
+    } else {
+      c0 = lane < m && gt0 < need_r && need_r <= ge0;
+      c1 = lane + 32 < m && gt1 < need_r && need_r <= ge1;
+    }
     const unsigned h0 = __ballot_sync(FULL, c0), h1 = __ballot_sync(FULL, c1);
-    if (!(h0 | h1)) { all = true; break; }       // cannot happen (1 <= need_r <= m)
+    if (!(h0 | h1)) { all = true; break; }       // cannot happen (the cut lies inside this bin)
     const int src = h0 ? __ffs(h0) - 1 : __ffs(h1) - 1;
     const float Tv = __shfl_sync(FULL, h0 ? a0 : a1, src);
     const int gt = __shfl_sync(FULL, h0 ? gt0 : gt1, src), ge = __shfl_sync(FULL, h0 ? ge0 : ge1, src);
-    T_lo = Tv; T_hi = Tv; need_t = need_r - gt; cnt_T = ge - gt;
+    T_lo = Tv; T_hi = Tv; cnt_T = ge - gt;
+    if constexpr (TOPP) {
+      const unsigned long long G = __shfl_sync(FULL, h0 ? G0 : G1, src), wT = __shfl_sync(FULL, h0 ? wa0 : wa1, src);
+      need_t = ties_for_mass(above_m + G, wT, cnt_T);
+    } else {
+      need_t = need_r - gt;
+    }
     break;
   }
 
@@ -1259,10 +1112,6 @@ k_select_topk(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack 
   for (int j = lane; j < g.NBt; j += 32)
     if (SPADE_CHECK(count + j < sh.cap, ws.status, 306, count + j)) out[count + j] = n + j;     // text KV blocks are always kept
   if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt;
-}
-
-inline size_t select_smem_bytes(const Shape& sh) {
-  return sizeof(float) * ((size_t)SEL_R * sh.ld_scores + (size_t)SEL_R * (sh.mode == 1 ? SEL_WARP_WORDS : SEL_WARP_WORDS - 512));
 }
 
 }  // namespace
@@ -1387,17 +1236,18 @@ cudaError_t launch_scores_minmax(const Shape& sh, const GeoPack& gp, const WsTab
 
 cudaError_t launch_select(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
                           cudaStream_t s) {
+  static_assert(SPADE_MAX_NB <= 16 * 128, "k_select_reg holds a row of at most 16 float4 per lane");
   dim3 grid((sh.NBmax + SEL_R - 1) / SEL_R, sh.BH);
-  if (sh.mode != 1 && sh.NBvmax <= 16 * 128) {          // Top-K with rows that fit the register file
-    if (sh.NBvmax <= 4 * 128) k_select_topk<4><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
-    else if (sh.NBvmax <= 8 * 128) k_select_topk<8><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
-    else if (sh.NBvmax <= 12 * 128) k_select_topk<12><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
-    else k_select_topk<16><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
-    return cudaGetLastError();
+  if (sh.mode != 1) {
+    if (sh.NBvmax <= 4 * 128) k_select_reg<4, false><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else if (sh.NBvmax <= 8 * 128) k_select_reg<8, false><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else if (sh.NBvmax <= 12 * 128) k_select_reg<12, false><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else k_select_reg<16, false><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+  } else {
+    if (sh.NBvmax <= 4 * 128) k_select_reg<4, true><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else if (sh.NBvmax <= 8 * 128) k_select_reg<8, true><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else if (sh.NBvmax <= 12 * 128) k_select_reg<12, true><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
+    else k_select_reg<16, true><<<grid, SEL_R * 32, 0, s>>>(sh, gp, st, ws);
   }
-  const size_t smem = select_smem_bytes(sh);
-  cudaError_t e = cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  k_select<<<grid, SEL_R * 32, smem, s>>>(sh, gp, st, ws);
   return cudaGetLastError();
 }

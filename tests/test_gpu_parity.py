@@ -137,16 +137,19 @@ def test_keep_one_and_keep_all():
     _run(base.replace(mode="topp", value=1.0))
 
 
-@pytest.mark.parametrize("grid,value", [((16, 32, 32), 0.8), ((16, 32, 32), 0.45), ((20, 32, 64), 0.8)])
-def test_topk_rows_with_ties_and_clusters_are_the_exact_top_k_lowest_ids_first(grid, value):
+@pytest.mark.parametrize("grid,mode,value", [((16, 32, 32), "sparsity", 0.8), ((16, 32, 32), "sparsity", 0.45), ((20, 32, 64), "sparsity", 0.8),
+                                             ((16, 32, 32), "topp", 0.5), ((20, 32, 64), "topp", 0.9)])
+def test_rows_with_ties_and_clusters_are_the_exact_top_of_the_table_lowest_ids_first(grid, mode, value):
     """Score rows that hold large groups of equal or nearly equal values (more than the 64 the index search ranks
     directly, so its histogram is refined between the group's own extremes, and rows where every score is the
-    same): the list must agree with the oracle away from the cut, and be the exact top-k of the fp32 table the
-    search read: nothing dropped scores higher than something kept, equal scores go by lower id."""
+    same): the list must agree with the oracle away from the cut, and be the exact top of the fp32 table the
+    search read: nothing dropped scores higher than something kept, equal scores go by lower id.  Top-K keeps
+    exactly k; Top-P keeps the shortest such prefix whose softmax mass reaches p (to 1e-4 of p: the search adds
+    the masses in 2^-40 fixed point)."""
     from tests import parity_util as pu
     from oracle import spade_oracle as so
     from paper_2608_03335_b200.workloads import make_qkv, bf16_bits
-    w = small_variant(WORKLOADS["wan14b"], heads=3, grid=grid).replace(mode="sparsity", value=value)
+    w = small_variant(WORKLOADS["wan14b"], heads=3, grid=grid).replace(mode=mode, value=value)
     blk = w.candidates[0]
     g = so.geometry(w.grid, w.n_text, blk)
     nbv = g["NBv"]
@@ -184,17 +187,30 @@ def test_topk_rows_with_ties_and_clusters_are_the_exact_top_k_lowest_ids_first(g
         big_groups = 0
         for bh in range(BH):
             S = t["block_scores"][bh, :nbv, :nbv].cpu().numpy()
-            k = int(keep[bh])
             for i in range(nbv):
                 kept = kv_idx[bh, i, :kv_cnt[bh, i]].tolist()
+                k = int(keep[bh]) if mode != "topp" else len(kept)
                 order = sorted(range(nbv), key=lambda j: (-S[i, j], j))
                 assert kept == sorted(order[:k]), f"head {bh} row {i}: not the top {k} by (score, lower id)"
+                if mode == "topp":
+                    wgt = np.exp(S[i, order].astype(np.float64) - float(S[i, order[0]]))
+                    run = np.cumsum(wgt) / wgt.sum()
+                    assert run[k - 1] >= value * (1 - 1e-4), f"head {bh} row {i}: kept mass {run[k - 1]} < p"
+                    assert k == 1 or run[k - 2] <= value * (1 + 1e-4), f"head {bh} row {i}: a shorter prefix holds {run[k - 2]}"
                 cut = S[i, order[k - 1]]
                 big_groups += int((np.abs(S[i] - cut) <= 1e-3 * max(abs(cut), 1e-6)).sum() > 64)
         assert big_groups > nbv, "the inputs did not put large groups at the cut"
-        print(f"[ties {grid} {value}] rows {rep.rows_checked} near-cut {rep.near_cut_blocks}, rows with > 64 values at the cut: {big_groups}")
+        print(f"[ties {grid} {mode} {value}] rows {rep.rows_checked} near-cut {rep.near_cut_blocks}, rows with > 64 values at the cut: {big_groups}")
     finally:
         plan.close()
+
+
+@pytest.mark.parametrize("mode,value", [("sparsity", 0.9), ("topp", 0.8)])
+def test_longest_rows_the_library_takes(mode, value):
+    """2048 video blocks per head, the most a plan accepts: the index search holds 16 float4 per lane, the
+    estimator walks 16 x 16 score tiles."""
+    w = small_variant(WORKLOADS["wan14b"], heads=1, grid=(32, 64, 64)).replace(mode=mode, value=value)
+    _run(w, forced=[0], rows_per_head=24, blocks_per_head=4, seed=17)
 
 
 def test_caller_written_lists_and_empty_rows():
