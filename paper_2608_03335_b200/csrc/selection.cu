@@ -245,11 +245,11 @@ k_static(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
 // Summaries of the chosen scheme, picked out of the all-candidate table of the block pass.
 __global__ void __launch_bounds__(256)
 k_gather(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws, const int split) {
-  const long total = (long)sh.BH * 2 * sh.NBmax * 32;       // float4 elements
-  for (long i = (long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long)gridDim.x * blockDim.x) {
-    const int c4 = (int)(i & 31);
-    const long rowi = i >> 5;
-    const int b = (int)(rowi % sh.NBmax), ht = (int)(rowi / sh.NBmax);
+  const unsigned total = (unsigned)sh.BH * 2u * (unsigned)sh.NBmax * 32u;       // float4 elements: at most 4096 * 2 * 2048 * 32 = 2^29
+  for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+    const int c4 = (int)(i & 31u);
+    const unsigned rowi = i >> 5;
+    const int b = (int)(rowi % (unsigned)sh.NBmax), ht = (int)(rowi / (unsigned)sh.NBmax);
     const int bh = ht >> 1, tensor = ht & 1;
     const int c = ws.scheme[bh];
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -470,11 +470,11 @@ __global__ void __launch_bounds__(1024) k_groups(const __grid_constant__ Shape s
 __global__ void __launch_bounds__(WARPS_PER_CTA * 32)
 k_pair_axis(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws) {
   const int lane = threadIdx.x & 31;
-  const long gw = (long)blockIdx.x * WARPS_PER_CTA + (threadIdx.x >> 5);
-  const long nw = (long)gridDim.x * WARPS_PER_CTA;
-  const long total = (long)sh.BH * 3 * sh.NBvmax;
-  for (long u = gw; u < total; u += nw) {
-    const int i = (int)(u % sh.NBvmax), axis = (int)((u / sh.NBvmax) % 3), bh = (int)(u / (3L * sh.NBvmax));
+  const int gw = blockIdx.x * WARPS_PER_CTA + (threadIdx.x >> 5);
+  const int nw = gridDim.x * WARPS_PER_CTA;
+  const int total = sh.BH * 3 * sh.NBvmax;            // at most 4096 * 3 * 2048
+  for (int u = gw; u < total; u += nw) {
+    const int i = u % sh.NBvmax, axis = (u / sh.NBvmax) % 3, bh = u / (3 * sh.NBvmax);
     const CandGeo& g = gp.g[ws.scheme[bh]];
     if (!g.pair || i >= g.NBv) continue;
     // a deterministic sample of about 400 blocks per head is enough to rank the three axes
@@ -819,6 +819,17 @@ k_select_reg(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack g
     if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = g.NB;
     return;
   }
+  uint32_t* bits = ws.rowbits + ((size_t)bh * sh.NBvmax + row) * sh.bits_ld;      // the same list as a bitmap, for k_pair_axis
+  if ((!TOPP && ws.keep[bh] >= n) || (sh.masks_on && ws.rowfull[(size_t)bh * sh.NBmax + row])) {
+    // every video block is kept: nothing to search, the scores are not read
+    for (int j = lane; j < n; j += 32)
+      if (SPADE_CHECK(j < sh.cap, ws.status, 302, j)) out[j] = j;
+    for (int wd = lane; wd * 32 < n; wd += 32) bits[wd] = n - wd * 32 >= 32 ? 0xffffffffu : (1u << (n - wd * 32)) - 1u;
+    for (int j = lane; j < g.NBt; j += 32)
+      if (SPADE_CHECK(n + j < sh.cap, ws.status, 306, n + j)) out[n + j] = n + j;
+    if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = n + g.NBt;
+    return;
+  }
   int* hcnt = sel_sm + warp * WORDS;                             // [256] bins, [256 + lane] dump slots, [288] list counter
   float* cand = reinterpret_cast<float*>(hcnt + 296);            // [SELR_CAND + 8]
   uint32_t* words = reinterpret_cast<uint32_t*>(hcnt + 296 + SELR_CAND + 8);     // [64] the row's keep bitmap
@@ -851,7 +862,7 @@ k_select_reg(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack g
 
   // ---- the cut: keep v > T_hi, and need_t of the cnt_T blocks with T_lo <= v <= T_hi (lowest ids first) ---------------
   int need_r = TOPP ? 1 : ws.keep[bh];                            // Top-K: blocks still to keep among those in [lo_v, hi_v]
-  bool all = !TOPP && need_r >= n;
+  bool all = false;                                               // set only if a pass finds its own histogram short (kept as a guard)
   int m = n;                                                      // blocks in [lo_v, hi_v]
   float T_lo = 0.f, T_hi = 0.f;
   int need_t = 0, cnt_T = 0;
@@ -1004,8 +1015,6 @@ k_select_reg(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack g
   }
 
   // ---- the keep bitmap, then the ascending id list ----------------------------------------------------------
-  if (sh.masks_on && ws.rowfull[(size_t)bh * sh.NBmax + row]) all = true;
-  uint32_t* bits = ws.rowbits + ((size_t)bh * sh.NBvmax + row) * sh.bits_ld;      // the same list as a bitmap, for k_pair_axis
   const int nw = (n + 31) >> 5;                  // <= NV * 4 <= 64 words
   if (all) {
     for (int wd = lane; wd < nw; wd += 32) words[wd] = n - wd * 32 >= 32 ? 0xffffffffu : (1u << (n - wd * 32)) - 1u;
