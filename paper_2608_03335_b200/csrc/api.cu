@@ -500,7 +500,7 @@ int spade_plan(spade_plan_t* p, const void* Q, const void* K, void* ws, void* st
     }
   }
   CUDA_TRY(launch_choose(p->sh, p->gp, p->st, t, fpack, skip_sics ? 0 : 1, s));
-  p->launches += 2;
+  p->launches += 1;
   if (p->sh.masks_on) {
     CUDA_TRY(launch_static(p->sh, p->gp, p->st, t, s));
     p->launches += 1;
@@ -562,12 +562,12 @@ int spade_select(spade_plan_t* p, void* ws, void* stream) {
   bool any_pair = false;
   for (int c = 0; c < p->sh.C; ++c) any_pair = any_pair || p->gp.g[c].pair;
   if (any_pair) {
-    // pair the 64-token query blocks along the axis that gives the shortest merged lists, per head
-    CUDA_TRY(cudaMemsetAsync(t.pair_union, 0, (size_t)p->sh.BH * 3 * 4, (cudaStream_t)stream));
+    // pair the 64-token query blocks along the axis that gives the shortest merged lists, per head (the totals start
+    // at zero: the plan stage and the previous use leave them so); the kernel's last CTA then orders the heads
     CUDA_TRY(launch_pair_axis(p->sh, p->gp, t, p->num_sms, (cudaStream_t)stream));
-    p->launches += 1;
+  } else {
+    CUDA_TRY(launch_groups_after_select(p->sh, p->gp, t, (cudaStream_t)stream));
   }
-  CUDA_TRY(launch_groups_after_select(p->sh, p->gp, t, (cudaStream_t)stream));
   p->launches += 1;
   p->stage = 3;
   return SPADE_OK;

@@ -328,6 +328,9 @@ k_split_k(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, 
 // One CTA per head: AS(X|c) = sum_b SICS (Eq. 3; fixed lane-strided order, one warp per (candidate, tensor)),
 // then warp 0: normalised score, argmax (ties -> lowest candidate) unless forced, and the head's keep count /
 // threshold.
+__device__ __forceinline__ void groups_body(const Shape& sh, const GeoPack& gp, const WsTables& ws, int mode);
+__device__ __forceinline__ bool last_cta_done(uint32_t* status, int word);
+
 __global__ void __launch_bounds__(256)
 k_choose(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws,
          const __grid_constant__ ForcedPack fp, int have_sics) {
@@ -345,7 +348,7 @@ k_choose(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
     }
   }
   __syncthreads();
-  if (warp != 0) return;
+  if (warp == 0) {
   int best = 0;
   if (have_sics) {
     float best_score = -1e30f;
@@ -378,6 +381,9 @@ k_choose(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
     ws.keep[bh] = keep;
     ws.pthr[bh] = p;
   }
+  }
+  // the last CTA to get here orders the heads for the attention kernel (what k_groups does in a launch of its own)
+  if (last_cta_done(ws.status, 9)) groups_body(sh, gp, ws, 0);
 }
 
 // Order in which the attention kernel takes the heads, heads per scheme, and the prefixes of attention
@@ -387,16 +393,18 @@ k_choose(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
 // mode 1 (after the index search): heads by decreasing list length per query tile, so that the longest
 // work items start first and the last ones are short; pairing axis = argmin of the merged-list totals
 // that k_pair_axis measured (ties -> w, then h, then t).
-__global__ void __launch_bounds__(1024) k_groups(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws, int mode) {
+// Runs in ONE CTA (every thread of it): k_groups, or the last CTA to finish of k_choose (mode 0) / k_pair_axis (mode 1).
+__device__ __forceinline__ void groups_body(const Shape& sh, const GeoPack& gp, const WsTables& ws, int mode) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nthreads = blockDim.x, nwarps = blockDim.x >> 5;
   if (tid == 0 && mode == 0 && sh.mode == 3) {
     // example policy function: keep fraction negatively correlated with the Selected Aggregation Score
     double abar = 0.0;
-    for (int bh = 0; bh < sh.BH; ++bh) abar += (double)ws.score[(size_t)bh * sh.C + ws.scheme[bh]];
+    for (int bh = 0; bh < sh.BH; ++bh) abar += (double)__ldcg(ws.score + (size_t)bh * sh.C + __ldcg(ws.scheme + bh));
     abar /= (double)sh.BH;
     for (int bh = 0; bh < sh.BH; ++bh) {
-      const int nkb = gp.g[ws.scheme[bh]].NBv;
-      const double a = (double)ws.score[(size_t)bh * sh.C + ws.scheme[bh]];
+      const int nkb = gp.g[__ldcg(ws.scheme + bh)].NBv;
+      const double a = (double)__ldcg(ws.score + (size_t)bh * sh.C + __ldcg(ws.scheme + bh));
       double f = (1.0 - (double)sh.value) * (1.0 - (double)sh.gain * (a - abar) / abar);
       f = f < 1.0 / nkb ? 1.0 / nkb : (f > 1.0 ? 1.0 : f);
       int k = (int)ceil(f * (double)nkb - 1e-9);
@@ -405,8 +413,8 @@ __global__ void __launch_bounds__(1024) k_groups(const __grid_constant__ Shape s
   }
   if (tid < SPADE_MAX_CANDS) ws.group_count[tid] = 0;
   // sort key per head (larger = earlier) and its pairing axis
-  for (int bh = warp; bh < sh.BH; bh += 32) {
-    const int c = ws.scheme[bh];
+  for (int bh = warp; bh < sh.BH; bh += nwarps) {
+    const int c = __ldcg(ws.scheme + bh);
     const CandGeo& g = gp.g[c];
     float key = -(float)c;
     if (mode == 1) {
@@ -423,23 +431,23 @@ __global__ void __launch_bounds__(1024) k_groups(const __grid_constant__ Shape s
     if (lane == 0) {
       int axis = 2;
       if (mode == 1 && g.pair) {
-        const int* u = ws.pair_union + bh * 3;
-        if (u[1] < u[axis]) axis = 1;
-        if (u[0] < u[axis]) axis = 0;
+        const int u0 = __ldcg(ws.pair_union + bh * 3), u1 = __ldcg(ws.pair_union + bh * 3 + 1), u2 = __ldcg(ws.pair_union + bh * 3 + 2);
+        if (u1 < u2) axis = 1;
+        if (u0 < (axis == 1 ? u1 : u2)) axis = 0;
       }
       ws.pair_axis[bh] = axis;
       ws.head_work[bh] = key;
     }
   }
   __syncthreads();
-  for (int i = tid; i < sh.BH; i += 1024) {                  // rank = heads that come before head i
+  for (int i = tid; i < sh.BH; i += nthreads) {                  // rank = heads that come before head i
     const float ki = ws.head_work[i];
     int rank = 0;
     for (int j = 0; j < sh.BH; ++j) {
       const float kj = ws.head_work[j];
       rank += (kj > ki || (kj == ki && j < i)) ? 1 : 0;
     }
-    const int c = ws.scheme[i];
+    const int c = __ldcg(ws.scheme + i);
     ws.head_order[rank] = i;
     ws.item_start[rank + 1] = head_tiles(gp.g[c], ws.pair_axis[i]);      // counts; scanned below
     ws.text_start[rank + 1] = gp.g[c].pair ? gp.g[c].ttiles : gp.g[c].NBt;
@@ -462,6 +470,29 @@ __global__ void __launch_bounds__(1024) k_groups(const __grid_constant__ Shape s
       carry_i = __shfl_sync(FULL, vi, 31); carry_t = __shfl_sync(FULL, vt, 31);
     }
   }
+  // the merged-list totals have been used (mode 1) or are not measured yet (mode 0): k_pair_axis adds into zeros
+  __syncthreads();
+  for (int i = tid; i < sh.BH * 3; i += nthreads) ws.pair_union[i] = 0;
+}
+
+__global__ void __launch_bounds__(1024) k_groups(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws, int mode) {
+  groups_body(sh, gp, ws, mode);
+}
+
+// True in every thread of the CTA that finishes last (a ticket in status word `word`, which the last CTA leaves at zero).
+// What the other CTAs wrote before their ticket is visible to it.
+__device__ __forceinline__ bool last_cta_done(uint32_t* status, int word) {
+  __shared__ int last_sm;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned ticket = atomicAdd(status + word, 1u);
+    last_sm = ticket == gridDim.x - 1 ? 1 : 0;
+    if (last_sm) status[word] = 0u;
+  }
+  __syncthreads();
+  if (last_sm) __threadfence();
+  return last_sm != 0;
 }
 
 // Merged-list length of a head's query tiles for each pairing axis (on a sample of the blocks): one warp
@@ -496,6 +527,8 @@ k_pair_axis(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp
     for (int o = 16; o >= 1; o >>= 1) uni += __shfl_xor_sync(FULL, uni, o);
     if (lane == 0) atomicAdd(&ws.pair_union[bh * 3 + axis], uni);
   }
+  // the last CTA to get here picks the axes and orders the heads by list length
+  if (last_cta_done(ws.status, 10)) groups_body(sh, gp, ws, 1);
 }
 
 // Mean summaries of the chosen scheme: one warp per (head, tensor, block).
@@ -1187,10 +1220,7 @@ cudaError_t launch_split_k(const Shape& sh, const GeoPack& gp, const WsTables& w
 
 cudaError_t launch_choose(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
                           const ForcedPack& forced, int have_sics, cudaStream_t s) {
-  k_choose<<<sh.BH, 256, 0, s>>>(sh, gp, st, ws, forced, have_sics);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  k_groups<<<1, 1024, 0, s>>>(sh, gp, ws, 0);
+  k_choose<<<sh.BH, 256, 0, s>>>(sh, gp, st, ws, forced, have_sics);      // its last CTA also orders the heads (k_groups, mode 0)
   return cudaGetLastError();
 }
 
