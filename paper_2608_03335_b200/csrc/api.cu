@@ -626,15 +626,35 @@ int spade_forward_host(spade_plan_t* p, const void* hQ, const void* hK, const vo
   // The AS-coupled budget needs the scores of all heads at once; everything else is per head.
   int chunks = p->sh.mode == SPADE_POLICY_AS ? 1 : (BH >= 32 ? 8 : BH >= 12 ? 6 : BH >= 4 ? 4 : 1);
   if (chunks > SPADE_HOST_CHUNKS) chunks = SPADE_HOST_CHUNKS;
-  const int per = (BH + chunks - 1) / chunks;
+  // The input copies are the slower side, so the kernels of a chunk always wait for its copy and the call ends
+  // one chunk's kernels and output copy after the last input byte: the last three chunks are small
+  // (3/40, 2/40 and 1/40 of the heads), the others share the rest evenly.
+  int size[SPADE_HOST_CHUNKS], first[SPADE_HOST_CHUNKS + 1];
+  {
+    int left = BH, n_small = chunks >= 6 ? 3 : 0;
+    for (int k = 0; k < n_small; ++k) {                  // sizes of the last chunks, the very last first
+      int sz = (BH * (k + 1) + 39) / 40;
+      sz = sz < 1 ? 1 : sz;
+      size[chunks - 1 - k] = sz;
+      left -= sz;
+    }
+    const int n_big = chunks - n_small;
+    for (int k = 0; k < n_big; ++k) {
+      const int sz = (left + (n_big - k) - 1) / (n_big - k);
+      size[k] = sz;
+      left -= sz;
+    }
+    first[0] = 0;
+    for (int k = 0; k < chunks; ++k) first[k + 1] = first[k] + size[k];
+  }
   const size_t head_bytes = (size_t)p->sh.N * SPADE_D * 2;
   // copies start after the work already queued on `stream` (it may still read the device buffers)
   CUDA_TRY(cudaEventRecord(p->ev_edge, s));
   CUDA_TRY(cudaStreamWaitEvent(p->copy_in, p->ev_edge, 0));
   CUDA_TRY(cudaStreamWaitEvent(p->copy_out, p->ev_edge, 0));
   int n_chunks = 0;
-  for (int h0 = 0; h0 < BH; h0 += per, ++n_chunks) {
-    const int nh = h0 + per <= BH ? per : BH - h0;
+  for (; n_chunks < chunks; ++n_chunks) {
+    const int h0 = first[n_chunks], nh = size[n_chunks];
     const size_t off = (size_t)h0 * head_bytes, bytes = (size_t)nh * head_bytes;
     CUDA_TRY(cudaMemcpyAsync((char*)dQ + off, (const char*)hQ + off, bytes, cudaMemcpyHostToDevice, p->copy_in));
     CUDA_TRY(cudaMemcpyAsync((char*)dK + off, (const char*)hK + off, bytes, cudaMemcpyHostToDevice, p->copy_in));
@@ -643,8 +663,8 @@ int spade_forward_host(spade_plan_t* p, const void* hQ, const void* hK, const vo
   }
   int launches = 0;
   rc = SPADE_OK;
-  for (int g = 0, h0 = 0; g < n_chunks && rc == SPADE_OK; ++g, h0 += per) {
-    const int nh = h0 + per <= BH ? per : BH - h0;
+  for (int g = 0; g < n_chunks && rc == SPADE_OK; ++g) {
+    const int h0 = first[g], nh = size[g];
     const size_t off = (size_t)h0 * head_bytes, bytes = (size_t)nh * head_bytes;
     spade_plan_s view = *p;                           // shares the static tables and the descriptor scratch
     view.sh.BH = nh;
