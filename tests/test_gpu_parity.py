@@ -454,7 +454,7 @@ def test_host_entry_point_matches_the_device_path(heads, pinned):
 
 
 def test_topp_one_keeps_the_mass_without_overrunning_the_histograms():
-    """p = 1: the crossing of the cumulative mass is decided by rounding; the radix descent must still
+    """p = 1: the crossing of the cumulative mass is decided by rounding; the histogram search must still
     land on a non-empty bin in every pass (regression: an empty bin left the next pass without keys)."""
     w = small_variant(WORKLOADS["wan14b"], heads=4, grid=(15, 18, 25)).replace(mode="topp", value=1.0)
     _run(w, forced=[0, 3, 2, 3], rows_per_head=40, blocks_per_head=4, seed=31)
@@ -545,7 +545,7 @@ def test_policy_budget_follows_the_aggregation_score():
 
 
 def test_topp_lists_are_reproducible_bit_for_bit_also_through_a_graph():
-    """The Top-P index search adds the softmax mass of a radix bin in fixed point, so the lists do not depend on
+    """The Top-P index search adds the softmax mass of a histogram bin in fixed point, so the lists do not depend on
     the order in which lanes reach a bin: two eager runs and two replays of a captured layer give identical
     kv_idx / kv_cnt (and outputs)."""
     from paper_2608_03335_b200 import binding
