@@ -54,7 +54,7 @@ struct WsLayout {
 
 }  // namespace
 
-#define SPADE_HOST_CHUNKS 8   // most head chunks spade_forward_host pipelines
+#define SPADE_HOST_CHUNKS 12  // most head chunks spade_forward_host pipelines
 
 struct spade_plan_s {
   int device, B, heads, num_sms;
@@ -624,28 +624,24 @@ int spade_forward_host(spade_plan_t* p, const void* hQ, const void* hK, const vo
   }
   const int BH = p->sh.BH;
   // The AS-coupled budget needs the scores of all heads at once; everything else is per head.
-  int chunks = p->sh.mode == SPADE_POLICY_AS ? 1 : (BH >= 32 ? 8 : BH >= 12 ? 6 : BH >= 4 ? 4 : 1);
+  int chunks = p->sh.mode == SPADE_POLICY_AS ? 1 : (BH >= 32 ? 12 : BH >= 12 ? 8 : BH >= 4 ? 4 : 1);
   if (chunks > SPADE_HOST_CHUNKS) chunks = SPADE_HOST_CHUNKS;
-  // The input copies are the slower side, so the kernels of a chunk always wait for its copy and the call ends
-  // one chunk's kernels and output copy after the last input byte: the last three chunks are small
-  // (3/40, 2/40 and 1/40 of the heads), the others share the rest evenly.
+  // The input copies are the slower side (about 1.1 ms per Wan-14B head against 0.9 ms of kernels), so the call ends one
+  // chunk's kernels and output copy after the last input byte, provided the kernels of chunk g are done by the time chunk
+  // g + 1 has arrived.  Chunk sizes therefore shrink geometrically, by a fifth from one chunk to the next.
   int size[SPADE_HOST_CHUNKS], first[SPADE_HOST_CHUNKS + 1];
   {
-    int left = BH, n_small = chunks >= 6 ? 3 : 0;
-    for (int k = 0; k < n_small; ++k) {                  // sizes of the last chunks, the very last first
-      int sz = (BH * (k + 1) + 39) / 40;
-      sz = sz < 1 ? 1 : sz;
-      size[chunks - 1 - k] = sz;
-      left -= sz;
-    }
-    const int n_big = chunks - n_small;
-    for (int k = 0; k < n_big; ++k) {
-      const int sz = (left + (n_big - k) - 1) / (n_big - k);
-      size[k] = sz;
-      left -= sz;
-    }
+    double w[SPADE_HOST_CHUNKS], total = 0.0, run = 0.0;
+    for (int k = 0; k < chunks; ++k) { w[k] = pow(1.25, (double)(chunks - 1 - k)); total += w[k]; }
     first[0] = 0;
-    for (int k = 0; k < chunks; ++k) first[k + 1] = first[k] + size[k];
+    for (int k = 0; k < chunks; ++k) {
+      run += w[k];
+      int end = k + 1 == chunks ? BH : (int)floor((double)BH * run / total + 0.5);
+      const int lo = first[k] + 1, hi = BH - (chunks - 1 - k);       // every chunk holds at least one head
+      end = end < lo ? lo : (end > hi ? hi : end);
+      first[k + 1] = end;
+      size[k] = end - first[k];
+    }
   }
   const size_t head_bytes = (size_t)p->sh.N * SPADE_D * 2;
   // copies start after the work already queued on `stream` (it may still read the device buffers)
