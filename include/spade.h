@@ -147,7 +147,7 @@ int spade_forward(spade_plan_t* plan, const void* Q, const void* K, const void* 
 
 /* End-to-end call with HOST tensors: copies hQ, hK, hV (host, same layout as the device tensors) into the
  * caller-provided device buffers dQ, dK, dV, runs the four stages, copies dO back into hO and returns
- * when all of it is done.  Heads are independent, so the call works on up to 8 chunks of heads and
+ * when all of it is done.  Heads are independent, so the call works on up to 12 chunks of heads (shrinking in size) and
  * overlaps the copies of one chunk with the kernels of another (two internal copy streams; the host
  * tensors must be pinned for the overlap, pageable memory still gives correct results).  Results are
  * identical to spade_forward on the same tensors.  SPADE_POLICY_AS budgets couple the heads and run as one

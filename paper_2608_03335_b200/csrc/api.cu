@@ -166,7 +166,7 @@ void compute_layout(spade_plan_s* p) {
   l.text_start = take((size_t)(BH + 1) * 4);
   l.kv_cnt = take((size_t)BH * sh.NBmax * 4);
   l.pair_axis = take((size_t)BH * 4);
-  l.pair_union = take((size_t)BH * 3 * 4);
+  l.pair_union = take((size_t)BH * 4 * 4);
   l.colkeep = take((size_t)BH * sh.NBmax);
   l.rowfull = take((size_t)BH * sh.NBmax);
   l.qsum = take((size_t)BH * sh.NBmax * SPADE_D * 4);

@@ -418,12 +418,7 @@ __device__ __forceinline__ void groups_body(const Shape& sh, const GeoPack& gp, 
     const CandGeo& g = gp.g[c];
     float key = -(float)c;
     if (mode == 1) {
-      const int* cnt = ws.kv_cnt + (size_t)bh * sh.NBmax;
-      int sum = 0;
-#pragma unroll 8
-      for (int r = lane; r < g.NBv; r += 32) sum += cnt[r];
-#pragma unroll
-      for (int o = 16; o >= 1; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+      const int sum = __ldcg(ws.pair_union + bh * 4 + 3);       // listed blocks over the head's video query rows (added up by the index search)
       // 64-key units per query tile, roughly: two per listed 128-token block; the merged list of two
       // 64-token query blocks is somewhat shorter than both lists together
       key = (float)sum / (float)g.NBv * (g.pair ? 1.7f : 2.0f);
@@ -431,7 +426,7 @@ __device__ __forceinline__ void groups_body(const Shape& sh, const GeoPack& gp, 
     if (lane == 0) {
       int axis = 2;
       if (mode == 1 && g.pair) {
-        const int u0 = __ldcg(ws.pair_union + bh * 3), u1 = __ldcg(ws.pair_union + bh * 3 + 1), u2 = __ldcg(ws.pair_union + bh * 3 + 2);
+        const int u0 = __ldcg(ws.pair_union + bh * 4), u1 = __ldcg(ws.pair_union + bh * 4 + 1), u2 = __ldcg(ws.pair_union + bh * 4 + 2);
         if (u1 < u2) axis = 1;
         if (u0 < (axis == 1 ? u1 : u2)) axis = 0;
       }
@@ -470,9 +465,9 @@ __device__ __forceinline__ void groups_body(const Shape& sh, const GeoPack& gp, 
       carry_i = __shfl_sync(FULL, vi, 31); carry_t = __shfl_sync(FULL, vt, 31);
     }
   }
-  // the merged-list totals have been used (mode 1) or are not measured yet (mode 0): k_pair_axis adds into zeros
+  // the per-head totals have been used (mode 1) or are not measured yet (mode 0): the index search and k_pair_axis add into zeros
   __syncthreads();
-  for (int i = tid; i < sh.BH * 3; i += nthreads) ws.pair_union[i] = 0;
+  for (int i = tid; i < sh.BH * 4; i += nthreads) ws.pair_union[i] = 0;
 }
 
 __global__ void __launch_bounds__(1024) k_groups(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws, int mode) {
@@ -525,7 +520,7 @@ k_pair_axis(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp
     for (int wd = lane; wd < words; wd += 32) uni += __popc(Bi[wd] | Bj[wd]);
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) uni += __shfl_xor_sync(FULL, uni, o);
-    if (lane == 0) atomicAdd(&ws.pair_union[bh * 3 + axis], uni);
+    if (lane == 0) atomicAdd(&ws.pair_union[bh * 4 + axis], uni);
   }
   // the last CTA to get here picks the axes and orders the heads by list length
   if (last_cta_done(ws.status, 10)) groups_body(sh, gp, ws, 1);
@@ -860,7 +855,7 @@ k_select_reg(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack g
     for (int wd = lane; wd * 32 < n; wd += 32) bits[wd] = n - wd * 32 >= 32 ? 0xffffffffu : (1u << (n - wd * 32)) - 1u;
     for (int j = lane; j < g.NBt; j += 32)
       if (SPADE_CHECK(n + j < sh.cap, ws.status, 306, n + j)) out[n + j] = n + j;
-    if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = n + g.NBt;
+    if (lane == 0) { ws.kv_cnt[(size_t)bh * sh.NBmax + row] = n + g.NBt; atomicAdd(&ws.pair_union[bh * 4 + 3], n + g.NBt); }
     return;
   }
   int* hcnt = sel_sm + warp * WORDS;                             // [256] bins, [256 + lane] dump slots, [288] list counter
@@ -1153,7 +1148,7 @@ k_select_reg(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack g
   const int count = tot0 + tot1;
   for (int j = lane; j < g.NBt; j += 32)
     if (SPADE_CHECK(count + j < sh.cap, ws.status, 306, count + j)) out[count + j] = n + j;     // text KV blocks are always kept
-  if (lane == 0) ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt;
+  if (lane == 0) { ws.kv_cnt[(size_t)bh * sh.NBmax + row] = count + g.NBt; atomicAdd(&ws.pair_union[bh * 4 + 3], count + g.NBt); }
 }
 
 }  // namespace

@@ -83,7 +83,7 @@ struct WsTables {
   float* csum;          // [BH][2 tensors][C][NBmax][128] mean summaries of every candidate
   float* nsum;          // same shape: sum over a block's tokens of q / |q| (one-pass scheme generation only)
   int* pair_axis;       // [BH] axis (0 t, 1 h, 2 w) along which 64-token query blocks are paired into 128-row tiles
-  int* pair_union;      // [BH][3] total merged-list length for each pairing axis
+  int* pair_union;      // [BH][4] total merged-list length for each pairing axis; [3] = blocks listed over the head's video query rows
   uint32_t* rowbits;    // [BH][NBvmax][bits_ld] the video part of every video query block's list as a bitmap (bit j = KV block j kept)
   uint8_t* colkeep;     // [BH][NBmax] KV block kept by every query block (intra rule on K, sink)
   uint8_t* rowfull;     // [BH][NBmax] query block keeps every block (intra rule on Q)
