@@ -416,7 +416,7 @@ def test_captured_layer_with_forced_schemes_keeps_them_after_the_host_list_is_go
         plan.close()
 
 
-@pytest.mark.parametrize("heads,pinned", [(5, True), (6, False), (9, True), (2, True)])
+@pytest.mark.parametrize("heads,pinned", [(5, True), (6, False), (9, True), (2, True), (13, True), (33, True)])
 def test_host_entry_point_matches_the_device_path(heads, pinned):
     """spade_forward_host (head chunks, copies overlapped with kernels) gives the bytes spade_forward gives."""
     from paper_2608_03335_b200 import binding
