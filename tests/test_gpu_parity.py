@@ -27,6 +27,15 @@ def test_tiny_topp():
     _run(WORKLOADS["tiny_topp"])
 
 
+@pytest.mark.parametrize("heads", [64, 200])
+def test_many_heads_on_a_tiny_grid(heads):
+    """More heads than the estimator has score tiles per SM: 64 heads give 64 tiles for 148 CTAs (ranges of zero
+    and one tile), 200 heads give ranges of one or two tiles that cross from one head into the next; the
+    plan-stage tables, the head ordering and the attention work list run with hundreds of heads as well."""
+    w = small_variant(WORKLOADS["wan14b"], heads=heads, grid=(4, 8, 16))
+    _run(w, rows_per_head=4, blocks_per_head=2, seed=23)
+
+
 def test_wan_small_ragged_grid_argmax_scheme():
     # 5x14x20: every candidate has partial edge blocks along some axis; odd block counts
     w = small_variant(WORKLOADS["wan1p3b"], heads=3, grid=(5, 14, 20))
