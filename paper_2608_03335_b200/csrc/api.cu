@@ -361,11 +361,13 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
   if (p->pf.on) {
     std::vector<int> pe;
     std::vector<float> pi;
-    plan_fused_tables(p->pf, sh, p->gp, pe, pi);
+    std::vector<uint32_t> pm;
+    plan_fused_tables(p->pf, sh, p->gp, pe, pi, pm);
     p->pf_entries = pe.size();
-    e = cudaMalloc(&p->d_pf, pe.size() * 8);
+    e = cudaMalloc(&p->d_pf, pe.size() * 8 + pm.size() * 4);
     if (e == cudaSuccess) e = cudaMemcpy(p->d_pf, pe.data(), pe.size() * 4, cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy((char*)p->d_pf + pe.size() * 4, pi.data(), pi.size() * 4, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy((char*)p->d_pf + pe.size() * 8, pm.data(), pm.size() * 4, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { cudaFree(p->d_pf); cudaFree(p->d_static); free(p); return fail(SPADE_ERR_CUDA, "table upload: %s", cudaGetErrorString(e)); }
   }
   compute_layout(p);
@@ -486,7 +488,8 @@ int spade_plan(spade_plan_t* p, const void* Q, const void* K, void* ws, void* st
         p->pq = Q; p->pk = K;
       }
       CUDA_TRY(launch_plan_fused(p->pmaps, Q, K, p->sh, p->gp, p->st, t, p->pf, p->num_sms, (const int*)p->d_pf,
-                                 (const float*)((const char*)p->d_pf + p->pf_entries * 4), s));
+                                 (const float*)((const char*)p->d_pf + p->pf_entries * 4),
+                                 (const uint32_t*)((const char*)p->d_pf + p->pf_entries * 8), s));
       p->launches += 2;
       p->have_csum = 1;
     } else if (p->sh.use_cells) {

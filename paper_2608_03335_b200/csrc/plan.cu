@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1)
 k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp,
              const WsTables ws, const __grid_constant__ PlanFusedCfg cfg,
              const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
-             const int* __restrict__ tab_e, const float* __restrict__ tab_inv) {
+             const int* __restrict__ tab_e, const float* __restrict__ tab_inv, const uint32_t* __restrict__ tab_m) {
   extern __shared__ __align__(1024) uint8_t pf_smem[];
   constexpr int NROWS = 32 * PF_NG * CPW;    // rows of the weight matrix = columns of D
   uint8_t* slices = pf_smem;                                            // cfg.stages x 32 KB
@@ -316,14 +316,17 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
             }
           }
           // Blocks that end at this slice are written.  Which of the warpgroup's slots end at (column, t), where
-          // their rows sit in the tables and the 1 / n of each block were worked out on the host: the whole
-          // output step is a table look-up and two predicated stores per slot, no branches.
+          // their rows sit in the tables and the 1 / n of each block were worked out on the host: the output
+          // step is a table look-up and two predicated stores per slot; a group of four slots none of which ends
+          // here (a bit mask per column, slice and warpgroup, the same for every thread) is skipped as a whole.
           {
             const size_t row = ((size_t)col * sh.T + t) * (PF_NG * 8 * CPW) + grp * (8 * CPW);
+            const uint32_t ends = __ldg(tab_m + ((size_t)col * sh.T + t) * PF_NG + grp);
             float* const cs = ws.csum + ((size_t)ht * sh.C * sh.NBmax) * SPADE_D + ch;
             float* const ns = ws.nsum + ((size_t)ht * sh.C * sh.NBmax) * SPADE_D + ch;
 #pragma unroll
             for (int k4 = 0; k4 < 8 * CPW; k4 += 4) {
+              if (!((ends >> k4) & 0xfu)) continue;
               const int4 e4 = __ldg(reinterpret_cast<const int4*>(tab_e + row + k4));
               const float4 i4 = __ldg(reinterpret_cast<const float4*>(tab_inv + row + k4));
               const int e[4] = {e4.x, e4.y, e4.z, e4.w};
@@ -480,10 +483,11 @@ int plan_encode_maps(PlanMaps* out, const void* Q, const void* K, const Shape& s
 // tables (candidate * NBmax + block id) if the block ends at slice t and lies inside the grid, else -1, and the
 // reciprocal of the block's valid-token count.  Slots are ordered [warpgroup][position] as the kernel reads them.
 void plan_fused_tables(const PlanFusedCfg& cfg, const Shape& sh, const GeoPack& gp, std::vector<int>& e,
-                       std::vector<float>& inv) {
+                       std::vector<float>& inv, std::vector<uint32_t>& ends) {
   const int ncol = cfg.ncol_h * cfg.ncol_w, per = PF_NG * 8 * cfg.cpw;
   e.assign((size_t)ncol * sh.T * per, -1);
   inv.assign((size_t)ncol * sh.T * per, 0.f);
+  ends.assign((size_t)ncol * sh.T * PF_NG, 0u);          // per (column, slice, warpgroup): bit k <=> the slot at position k ends here
   for (int col = 0; col < ncol; ++col) {
     const int ch0 = (col / cfg.ncol_w) * cfg.colH, cw0 = (col % cfg.ncol_w) * cfg.colW;
     for (int t = 0; t < sh.T; ++t)
@@ -500,6 +504,7 @@ void plan_fused_tables(const PlanFusedCfg& cfg, const Shape& sh, const GeoPack& 
         const int nw = g.bw < sh.W - iw * g.bw ? g.bw : sh.W - iw * g.bw;
         const size_t at = ((size_t)col * sh.T + t) * per + (j % PF_NG) * (8 * cfg.cpw) + j / PF_NG;
         e[at] = c * sh.NBmax + (it * g.nbh + ih) * g.nbw + iw;
+        ends[((size_t)col * sh.T + t) * PF_NG + j % PF_NG] |= 1u << (j / PF_NG);
         inv[at] = 1.f / (float)(nt * nh * nw);
       }
   }
@@ -507,7 +512,7 @@ void plan_fused_tables(const PlanFusedCfg& cfg, const Shape& sh, const GeoPack& 
 
 cudaError_t launch_plan_fused(const PlanMaps* maps, const void* Q, const void* K, const Shape& sh, const GeoPack& gp,
                               const StaticTables& st, const WsTables& ws, const PlanFusedCfg& cfg, int num_sms,
-                              const int* tab_e, const float* tab_inv, cudaStream_t s) {
+                              const int* tab_e, const float* tab_inv, const uint32_t* tab_m, cudaStream_t s) {
   (void)st;
   const size_t smem = plan_fused_smem(cfg);
   const long items = (long)sh.BH * 2 * cfg.nchunks * cfg.ncol_h * cfg.ncol_w;
@@ -519,7 +524,7 @@ cudaError_t launch_plan_fused(const PlanMaps* maps, const void* Q, const void* K
     e = cudaFuncSetAttribute(k_plan_fused<CPW_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);            \
     if (e != cudaSuccess) return e;                                                                                  \
     k_plan_fused<CPW_><<<(unsigned)grid, PF_THREADS, smem, s>>>(*maps, sh, gp, ws, cfg, (const __nv_bfloat16*)Q,     \
-                                                                (const __nv_bfloat16*)K, tab_e, tab_inv);           \
+                                                                (const __nv_bfloat16*)K, tab_e, tab_inv, tab_m);    \
   }
   PF_LAUNCH(1) PF_LAUNCH(2) PF_LAUNCH(3) PF_LAUNCH(4)
 #undef PF_LAUNCH

@@ -174,10 +174,10 @@ void plan_fused_configure(PlanFusedCfg* cfg, const Shape& sh, const GeoPack& gp,
 int plan_encode_maps(PlanMaps* out, const void* Q, const void* K, const Shape& sh, const PlanFusedCfg& cfg, char* err,
                      size_t errlen);
 void plan_fused_tables(const PlanFusedCfg& cfg, const Shape& sh, const GeoPack& gp, std::vector<int>& e,
-                       std::vector<float>& inv);
+                       std::vector<float>& inv, std::vector<uint32_t>& ends);
 cudaError_t launch_plan_fused(const PlanMaps* maps, const void* Q, const void* K, const Shape& sh, const GeoPack& gp,
                               const StaticTables& st, const WsTables& ws, const PlanFusedCfg& cfg, int num_sms,
-                              const int* tab_e, const float* tab_inv, cudaStream_t s);
+                              const int* tab_e, const float* tab_inv, const uint32_t* tab_m, cudaStream_t s);
 
 struct ScoreMaps;  // tensor map of the K' summaries, defined in scores.cu
 size_t score_maps_bytes();
