@@ -72,9 +72,26 @@ __device__ __forceinline__ uint32_t pf_w_offset(int nrows, int n, int tok) {
 // Row of the weight matrix (= column of D) of (slot, piece).  Slots go round the four epilogue warpgroups
 // (slot mod 4), so that the candidates whose blocks end most often are shared by all; a warpgroup's slots
 // sit in CPW chunks of 32 columns, 8 slots of 4 pieces each.
+// Two slots share eight columns, piece by piece: [r1 a, r1 b, r2 a, r2 b, r3 a, r3 b, ones a, ones b], so that the
+// epilogue adds the pieces of both with packed fp32 instructions on adjacent registers.
 __device__ __forceinline__ int pf_row(int cpw, int slot, int piece) {
   const int k = slot / PF_NG;
-  return 32 * ((slot % PF_NG) * cpw + (k >> 3)) + 4 * (k & 7) + piece;
+  return 32 * ((slot % PF_NG) * cpw + (k >> 3)) + 8 * ((k & 7) >> 1) + 2 * piece + (k & 1);
+}
+__device__ __forceinline__ uint64_t pf_pack2(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t pf_add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float pf_half(uint64_t v, int hi) {
+  float a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+  return hi ? b : a;
 }
 
 template <int CPW>
@@ -293,9 +310,9 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
       const int wq = warp & 3;
       const int ch = wq * 32 + lane;
       const uint32_t lane_base = (uint32_t)(wq * 32) << 16;
-      float an[8 * CPW], ar[8 * CPW];
+      uint64_t an[4 * CPW], ar[4 * CPW];       // per pair of slots (2p, 2p + 1): summed q / |q| and summed q of this channel, packed fp32 x 2
 #pragma unroll
-      for (int k = 0; k < 8 * CPW; ++k) an[k] = ar[k] = 0.f;
+      for (int k = 0; k < 4 * CPW; ++k) an[k] = ar[k] = 0ull;
       uint32_t i = 0;
       for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
         const int col = item % col_items, chunk = (item / col_items) % cfg.nchunks, ht = item / (col_items * cfg.nchunks);
@@ -310,9 +327,10 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
             ptx::tmem_ld32(tmem_D + lane_base + b * NROWS + (grp * CPW + q) * 32, r);
             ptx::tmem_wait_ld();
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              an[q * 8 + k] += (__uint_as_float(r[4 * k]) + __uint_as_float(r[4 * k + 1])) + __uint_as_float(r[4 * k + 2]);
-              ar[q * 8 + k] += __uint_as_float(r[4 * k + 3]);
+            for (int pr = 0; pr < 4; ++pr) {
+              const uint64_t p12 = pf_add2(pf_pack2(r[8 * pr], r[8 * pr + 1]), pf_pack2(r[8 * pr + 2], r[8 * pr + 3]));
+              an[q * 4 + pr] = pf_add2(an[q * 4 + pr], pf_add2(p12, pf_pack2(r[8 * pr + 4], r[8 * pr + 5])));
+              ar[q * 4 + pr] = pf_add2(ar[q * 4 + pr], pf_pack2(r[8 * pr + 6], r[8 * pr + 7]));
             }
           }
           // Blocks that end at this slice are written.  Which of the warpgroup's slots end at (column, t), where
@@ -334,12 +352,15 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
                 const int k = k4 + u;
+                const float anv = pf_half(an[k >> 1], k & 1), arv = pf_half(ar[k >> 1], k & 1);
                 if (e[u] >= 0 && SPADE_CHECK(e[u] < sh.C * sh.NBmax, ws.status, 601, e[u])) {
-                  cs[(size_t)e[u] * SPADE_D] = ar[k] * iv[u];          // mean summary, this channel
-                  ns[(size_t)e[u] * SPADE_D] = an[k];                  // sum of q / |q|; SICS = its squared norm
+                  cs[(size_t)e[u] * SPADE_D] = arv * iv[u];            // mean summary, this channel
+                  ns[(size_t)e[u] * SPADE_D] = anv;                    // sum of q / |q|; SICS = its squared norm
                 }
-                an[k] = e[u] >= 0 ? 0.f : an[k];
-                ar[k] = e[u] >= 0 ? 0.f : ar[k];
+                if (e[u] >= 0) {                                       // the block is done: its half of the pair starts again at zero
+                  an[k >> 1] = (k & 1) ? pf_pack2(__float_as_uint(pf_half(an[k >> 1], 0)), 0u) : pf_pack2(0u, __float_as_uint(pf_half(an[k >> 1], 1)));
+                  ar[k >> 1] = (k & 1) ? pf_pack2(__float_as_uint(pf_half(ar[k >> 1], 0)), 0u) : pf_pack2(0u, __float_as_uint(pf_half(ar[k >> 1], 1)));
+                }
               }
             }
           }
