@@ -175,9 +175,9 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
         const int t0 = chunk * cfg.tchunk, t1 = min(sh.T, t0 + cfg.tchunk);
         for (int t = t0; t < t1; ++t, ++i) {
           const uint32_t s = i % cfg.stages, b = i & 1, ph = (i >> 1) & 1;
-          if (!ptx::mbar_wait_sleepy(&ctl.full[s], (i / cfg.stages) & 1, &ctl.abort, PF_WAIT_NS) ||
-              !ptx::mbar_wait_sleepy(&ctl.w_full[b], ph, &ctl.abort, PF_WAIT_NS) ||
-              !ptx::mbar_wait_sleepy(&ctl.d_empty[b], ph ^ 1, &ctl.abort, PF_WAIT_NS)) { site = 205; break; }
+          if (!ptx::mbar_wait(&ctl.full[s], (i / cfg.stages) & 1, &ctl.abort, PF_WAIT_NS) ||
+              !ptx::mbar_wait(&ctl.w_full[b], ph, &ctl.abort, PF_WAIT_NS) ||
+              !ptx::mbar_wait(&ctl.d_empty[b], ph ^ 1, &ctl.abort, PF_WAIT_NS)) { site = 205; break; }
           ptx::tc_fence_after();
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {        // 16 tokens per step
@@ -319,7 +319,7 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
         const int t0 = chunk * cfg.tchunk, t1 = min(sh.T, t0 + cfg.tchunk);
         for (int t = t0; t < t1 && !site; ++t, ++i) {
           const uint32_t b = i & 1, ph = (i >> 1) & 1;
-          if (!ptx::mbar_wait_warp(&ctl.d_full[b], ph, &ctl.abort, PF_WAIT_NS)) { site = 207; break; }
+          if (!__all_sync(FULL, ptx::mbar_wait(&ctl.d_full[b], ph, &ctl.abort, PF_WAIT_NS))) { site = 207; break; }
           ptx::tc_fence_after();
 #pragma unroll
           for (int q = 0; q < CPW; ++q) {
