@@ -169,7 +169,7 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
         site_item = it.bh * 4096 + it.rt;
         for (int e = 0; e < 2 + 4 * it.n_ct; ++e, ++ent) {
           const uint32_t st = ent % SC_NST;
-          if (!ptx::mbar_wait_sleepy(&ctl.empty[st], ((ent / SC_NST) & 1) ^ 1, &ctl.abort, SC_WAIT_NS)) { site = 101; break; }
+          if (!ptx::mbar_wait(&ctl.empty[st], ((ent / SC_NST) & 1) ^ 1, &ctl.abort, SC_WAIT_NS)) { site = 101; break; }
           uint8_t* dst = smem + st * SC_ENTRY;
           ptx::mbar_expect_tx(&ctl.full[st], SC_ENTRY);
           if (e < 2) {
@@ -237,7 +237,7 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
 
     auto epilogue = [&](int bh, int rt, int ctile, int nbv, uint32_t tt) -> bool {
       const uint32_t sp = tt & 1;
-      if (!ptx::mbar_wait_warp(&ctl.mma_done[sp], (tt >> 1) & 1, &ctl.abort, SC_WAIT_NS)) return false;
+      if (!__all_sync(0xffffffffu, ptx::mbar_wait(&ctl.mma_done[sp], (tt >> 1) & 1, &ctl.abort, SC_WAIT_NS))) return false;
       ptx::tc_fence_after();
       const bool rows_live = rt * 128 + warp * 32 < nbv;      // none of this warp's 32 rows is a video block otherwise
 #pragma unroll 1
@@ -278,7 +278,7 @@ k_scores(const __grid_constant__ ScoreMaps maps, const __grid_constant__ Shape s
       if (!ptx::mbar_wait_warp(&ctl.full[st0], (ent / SC_NST) & 1, &ctl.abort, SC_WAIT_NS) ||
           !ptx::mbar_wait_warp(&ctl.full[st1], ((ent + 1) / SC_NST) & 1, &ctl.abort, SC_WAIT_NS)) { site = 105; break; }
       // every product that reads the previous A is complete once the previous item's last tile is
-      if (pend_bh >= 0 && !ptx::mbar_wait_warp(&ctl.mma_done[pend_tile & 1], (pend_tile >> 1) & 1, &ctl.abort, SC_WAIT_NS)) { site = 106; break; }
+      if (pend_bh >= 0 && !__all_sync(0xffffffffu, ptx::mbar_wait(&ctl.mma_done[pend_tile & 1], (pend_tile >> 1) & 1, &ctl.abort, SC_WAIT_NS))) { site = 106; break; }
       ptx::tc_fence_after();
 #pragma unroll 1
       for (int g = 0; g < 4; ++g) {                     // 32 channels per step
