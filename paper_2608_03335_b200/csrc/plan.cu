@@ -48,6 +48,7 @@ constexpr int PF_WARP_LOAD = 4 + 4 * PF_NG, PF_WARP_MMA = PF_WARP_LOAD + 1;
 struct PfCtl {
   uint64_t full[PF_MAX_STAGES], empty[PF_MAX_STAGES];
   uint64_t w_full[2], w_empty[2], d_full[2], d_empty[2];
+  uint64_t tab_full[2], tab_empty[2];      // the output table rows of a work item in shared memory (loader -> epilogue warps)
   uint32_t tmem_base;
   volatile uint32_t abort;
   float sp[2][64][4];        // SICS partials of the four warps of a warpgroup, per slice parity and slot
@@ -106,7 +107,11 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
   uint8_t* wmat = pf_smem + cfg.stages * PF_SLICE_BYTES;                // 2 buffers x (2 halves x NROWS x 128 B)
   constexpr int W_BYTES = 2 * NROWS * 128;
   constexpr uint32_t TMEM_COLS = 2 * NROWS <= 128 ? 128 : 2 * NROWS <= 256 ? 256 : 512;     // a power of two
-  PfCtl& ctl = *reinterpret_cast<PfCtl*>(wmat + 2 * W_BYTES);
+  // per work item: tchunk rows of the row table, of the 1/n table and of the end masks (16 bytes per slice), two buffers
+  constexpr int PER = PF_NG * 8 * CPW;
+  const int TAB_BYTES = cfg.tchunk * (PER * 8 + 16);
+  uint8_t* tabs = wmat + 2 * W_BYTES;
+  PfCtl& ctl = *reinterpret_cast<PfCtl*>(tabs + 2 * TAB_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int col_items = cfg.ncol_h * cfg.ncol_w;
   const int items = sh.BH * 2 * cfg.nchunks * col_items;
@@ -117,6 +122,7 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(&ctl.w_full[b], 4); ptx::mbar_init(&ctl.w_empty[b], 1);
       ptx::mbar_init(&ctl.d_full[b], 1); ptx::mbar_init(&ctl.d_empty[b], 4 * PF_NG);
+      ptx::mbar_init(&ctl.tab_full[b], 1); ptx::mbar_init(&ctl.tab_empty[b], 4 * PF_NG);
     }
     ctl.abort = 0;
     ptx::fence_mbar_init();
@@ -149,12 +155,23 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
   if (warp == PF_WARP_LOAD) {
     // ================= loader: slices of this CTA's work items through the ring ==========================
     if (lane == 0) {
-      uint32_t i = 0;
+      uint32_t i = 0, nit = 0;
       for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
         const int col = item % col_items, chunk = (item / col_items) % cfg.nchunks, ht = item / (col_items * cfg.nchunks);
         const int h0 = (col / cfg.ncol_w) * cfg.colH, w0 = (col % cfg.ncol_w) * cfg.colW;
         const int t0 = chunk * cfg.tchunk, t1 = min(sh.T, t0 + cfg.tchunk);
         const CUtensorMap* map = (ht & 1) ? &maps.k : &maps.q;
+        {                                         // the item's rows of the output tables, ahead of its slices
+          const uint32_t tb = nit & 1, nsl = (uint32_t)(t1 - t0);
+          if (!ptx::mbar_wait_sleepy(&ctl.tab_empty[tb], ((nit >> 1) & 1) ^ 1, &ctl.abort, PF_WAIT_NS)) { site = 203; break; }
+          uint8_t* dst = tabs + tb * TAB_BYTES;
+          const size_t r0 = (size_t)col * sh.T + t0;
+          ptx::mbar_expect_tx(&ctl.tab_full[tb], nsl * (PER * 8 + 16));
+          ptx::bulk_load(dst, tab_e + r0 * PER, nsl * PER * 4, &ctl.tab_full[tb]);
+          ptx::bulk_load(dst + cfg.tchunk * PER * 4, tab_inv + r0 * PER, nsl * PER * 4, &ctl.tab_full[tb]);
+          ptx::bulk_load(dst + cfg.tchunk * PER * 8, tab_m + r0 * 4, nsl * 16, &ctl.tab_full[tb]);
+          ++nit;
+        }
         for (int t = t0; t < t1; ++t, ++i) {
           const uint32_t s = i % cfg.stages, par = ((i / cfg.stages) & 1) ^ 1;
           if (!ptx::mbar_wait_sleepy(&ctl.empty[s], par, &ctl.abort, PF_WAIT_NS)) { site = 201; break; }
@@ -313,10 +330,17 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
       uint64_t an[4 * CPW], ar[4 * CPW];       // per pair of slots (2p, 2p + 1): summed q / |q| and summed q of this channel, packed fp32 x 2
 #pragma unroll
       for (int k = 0; k < 4 * CPW; ++k) an[k] = ar[k] = 0ull;
-      uint32_t i = 0;
-      for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
-        const int col = item % col_items, chunk = (item / col_items) % cfg.nchunks, ht = item / (col_items * cfg.nchunks);
+      uint32_t i = 0, nit = 0;
+      for (int item = blockIdx.x; item < items && !site; item += gridDim.x, ++nit) {
+        const int chunk = (item / col_items) % cfg.nchunks, ht = item / (col_items * cfg.nchunks);
         const int t0 = chunk * cfg.tchunk, t1 = min(sh.T, t0 + cfg.tchunk);
+        // the item's rows of the output tables arrive in shared memory (a row is used once: from global memory every
+        // slice paid two trips to the L2 in the middle of its output step)
+        const uint32_t tb = nit & 1;
+        if (!__all_sync(FULL, ptx::mbar_wait(&ctl.tab_full[tb], (nit >> 1) & 1, &ctl.abort, PF_WAIT_NS))) { site = 209; break; }
+        const int* const s_e = reinterpret_cast<const int*>(tabs + tb * TAB_BYTES) + grp * (8 * CPW);
+        const float* const s_inv = reinterpret_cast<const float*>(tabs + tb * TAB_BYTES + cfg.tchunk * PER * 4) + grp * (8 * CPW);
+        const uint32_t* const s_m = reinterpret_cast<const uint32_t*>(tabs + tb * TAB_BYTES + cfg.tchunk * PER * 8) + grp;
         for (int t = t0; t < t1 && !site; ++t, ++i) {
           const uint32_t b = i & 1, ph = (i >> 1) & 1;
           if (!__all_sync(FULL, ptx::mbar_wait(&ctl.d_full[b], ph, &ctl.abort, PF_WAIT_NS))) { site = 207; break; }
@@ -338,15 +362,15 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
           // step is a table look-up and two predicated stores per slot; a group of four slots none of which ends
           // here (a bit mask per column, slice and warpgroup, the same for every thread) is skipped as a whole.
           {
-            const size_t row = ((size_t)col * sh.T + t) * (PF_NG * 8 * CPW) + grp * (8 * CPW);
-            const uint32_t ends = __ldg(tab_m + ((size_t)col * sh.T + t) * PF_NG + grp);
+            const int row = (t - t0) * PER;
+            const uint32_t ends = s_m[(t - t0) * 4];
             float* const cs = ws.csum + ((size_t)ht * sh.C * sh.NBmax) * SPADE_D + ch;
             float* const ns = ws.nsum + ((size_t)ht * sh.C * sh.NBmax) * SPADE_D + ch;
 #pragma unroll
             for (int k4 = 0; k4 < 8 * CPW; k4 += 4) {
               if (!((ends >> k4) & 0xfu)) continue;
-              const int4 e4 = __ldg(reinterpret_cast<const int4*>(tab_e + row + k4));
-              const float4 i4 = __ldg(reinterpret_cast<const float4*>(tab_inv + row + k4));
+              const int4 e4 = *reinterpret_cast<const int4*>(s_e + row + k4);
+              const float4 i4 = *reinterpret_cast<const float4*>(s_inv + row + k4);
               const int e[4] = {e4.x, e4.y, e4.z, e4.w};
               const float iv[4] = {i4.x, i4.y, i4.z, i4.w};
 #pragma unroll
@@ -368,6 +392,8 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&ctl.d_empty[b]);           // after the outputs: keeps the warps within two slices
         }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&ctl.tab_empty[tb]);          // the table buffer may take the item after next
       }
     }
   }
@@ -433,7 +459,7 @@ EncodeFn encode_fn() {
 }
 
 size_t plan_fused_smem(const PlanFusedCfg& cfg) {
-  return (size_t)cfg.stages * PF_SLICE_BYTES + (size_t)2 * (2 * cfg.nrows * 128) + sizeof(PfCtl);
+  return (size_t)cfg.stages * PF_SLICE_BYTES + (size_t)2 * (2 * cfg.nrows * 128) + (size_t)2 * cfg.tchunk * (PF_NG * 8 * cfg.cpw * 8 + 16) + sizeof(PfCtl);
 }
 
 int ilog2(int x) { int l = 0; while ((1 << l) < x) ++l; return l; }
@@ -508,7 +534,7 @@ void plan_fused_tables(const PlanFusedCfg& cfg, const Shape& sh, const GeoPack& 
   const int ncol = cfg.ncol_h * cfg.ncol_w, per = PF_NG * 8 * cfg.cpw;
   e.assign((size_t)ncol * sh.T * per, -1);
   inv.assign((size_t)ncol * sh.T * per, 0.f);
-  ends.assign((size_t)ncol * sh.T * PF_NG, 0u);          // per (column, slice, warpgroup): bit k <=> the slot at position k ends here
+  ends.assign((size_t)ncol * sh.T * 4, 0u);              // per (column, slice): one word per warpgroup (16 bytes per slice), bit k <=> the slot at position k ends here
   for (int col = 0; col < ncol; ++col) {
     const int ch0 = (col / cfg.ncol_w) * cfg.colH, cw0 = (col % cfg.ncol_w) * cfg.colW;
     for (int t = 0; t < sh.T; ++t)
@@ -525,7 +551,7 @@ void plan_fused_tables(const PlanFusedCfg& cfg, const Shape& sh, const GeoPack& 
         const int nw = g.bw < sh.W - iw * g.bw ? g.bw : sh.W - iw * g.bw;
         const size_t at = ((size_t)col * sh.T + t) * per + (j % PF_NG) * (8 * cfg.cpw) + j / PF_NG;
         e[at] = c * sh.NBmax + (it * g.nbh + ih) * g.nbw + iw;
-        ends[((size_t)col * sh.T + t) * PF_NG + j % PF_NG] |= 1u << (j / PF_NG);
+        ends[((size_t)col * sh.T + t) * 4 + j % PF_NG] |= 1u << (j / PF_NG);
         inv[at] = 1.f / (float)(nt * nh * nw);
       }
   }
