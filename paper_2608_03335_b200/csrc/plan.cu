@@ -155,7 +155,7 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
   if (warp == PF_WARP_LOAD) {
     // ================= loader: slices of this CTA's work items through the ring ==========================
     if (lane == 0) {
-      uint32_t i = 0, nit = 0;
+      uint32_t nit = 0, s = 0, sph = 0;          // ring stage of the next slice and its phase (kept by hand: a division per slice costs a single thread hundreds of cycles)
       for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
         const int col = item % col_items, chunk = (item / col_items) % cfg.nchunks, ht = item / (col_items * cfg.nchunks);
         const int h0 = (col / cfg.ncol_w) * cfg.colH, w0 = (col % cfg.ncol_w) * cfg.colW;
@@ -172,12 +172,12 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
           ptx::bulk_load(dst + cfg.tchunk * PER * 8, tab_m + r0 * 4, nsl * 16, &ctl.tab_full[tb]);
           ++nit;
         }
-        for (int t = t0; t < t1; ++t, ++i) {
-          const uint32_t s = i % cfg.stages, par = ((i / cfg.stages) & 1) ^ 1;
-          if (!ptx::mbar_wait_sleepy(&ctl.empty[s], par, &ctl.abort, PF_WAIT_NS)) { site = 201; break; }
+        for (int t = t0; t < t1; ++t) {
+          if (!ptx::mbar_wait_sleepy(&ctl.empty[s], sph ^ 1, &ctl.abort, PF_WAIT_NS)) { site = 201; break; }
           ptx::mbar_expect_tx(&ctl.full[s], PF_SLICE_BYTES);
           ptx::tma_load_5d(slices + s * PF_SLICE_BYTES, map, &ctl.full[s], 0, w0, h0, t, ht >> 1);
           ptx::tma_load_5d(slices + s * PF_SLICE_BYTES + PF_HALF_BYTES, map, &ctl.full[s], 64, w0, h0, t, ht >> 1);
+          if (++s == (uint32_t)cfg.stages) { s = 0; sph ^= 1; }
         }
       }
     }
@@ -186,13 +186,13 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
     if (lane == 0) {
       const uint32_t idesc = pf_idesc(128, NROWS);
       const uint32_t aS = ptx::smem_u32(slices), aW = ptx::smem_u32(wmat);
-      uint32_t i = 0;
+      uint32_t i = 0, s = 0, sph = 0;        // slice count; ring stage and its phase
       for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
         const int chunk = (item / col_items) % cfg.nchunks;
         const int t0 = chunk * cfg.tchunk, t1 = min(sh.T, t0 + cfg.tchunk);
         for (int t = t0; t < t1; ++t, ++i) {
-          const uint32_t s = i % cfg.stages, b = i & 1, ph = (i >> 1) & 1;
-          if (!ptx::mbar_wait(&ctl.full[s], (i / cfg.stages) & 1, &ctl.abort, PF_WAIT_NS) ||
+          const uint32_t b = i & 1, ph = (i >> 1) & 1;
+          if (!ptx::mbar_wait(&ctl.full[s], sph, &ctl.abort, PF_WAIT_NS) ||
               !ptx::mbar_wait(&ctl.w_full[b], ph, &ctl.abort, PF_WAIT_NS) ||
               !ptx::mbar_wait(&ctl.d_empty[b], ph ^ 1, &ctl.abort, PF_WAIT_NS)) { site = 205; break; }
           ptx::tc_fence_after();
@@ -205,6 +205,7 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
           ptx::umma_commit(&ctl.d_full[b]);
           ptx::umma_commit(&ctl.w_empty[b]);
           ptx::umma_commit(&ctl.empty[s]);
+          if (++s == (uint32_t)cfg.stages) { s = 0; sph ^= 1; }
         }
       }
     }
@@ -220,13 +221,13 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
 #pragma unroll
       for (int pce = 0; pce < 3; ++pce) woff[c][pce] = pf_w_offset(NROWS, pf_row(CPW, slot, pce), tok);
     }
-    uint32_t i = 0;
+    uint32_t i = 0, s = 0, sph = 0;
     for (int item = blockIdx.x; item < items && !site; item += gridDim.x) {
       const int chunk = (item / col_items) % cfg.nchunks;
       const int t0 = chunk * cfg.tchunk, t1 = min(sh.T, t0 + cfg.tchunk);
       for (int t = t0; t < t1 && !site; ++t, ++i) {
-        const uint32_t s = i % cfg.stages, b = i & 1, ph = (i >> 1) & 1;
-        if (!ptx::mbar_wait_warp(&ctl.full[s], (i / cfg.stages) & 1, &ctl.abort, PF_WAIT_NS)) { site = 202; break; }
+        const uint32_t b = i & 1, ph = (i >> 1) & 1;
+        if (!ptx::mbar_wait_warp(&ctl.full[s], sph, &ctl.abort, PF_WAIT_NS)) { site = 202; break; }
         const uint8_t* row = slices + s * PF_SLICE_BYTES + tok * 128;
         uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
@@ -281,6 +282,7 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
         ptx::fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ctl.w_full[b]);
+        if (++s == (uint32_t)cfg.stages) { s = 0; sph ^= 1; }
       }
     }
     // ---- text blocks (outside the 3-D grid: no SICS, mean summaries only), straight from their rows ------
