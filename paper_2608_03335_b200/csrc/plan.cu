@@ -359,6 +359,10 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
               ar[q * 4 + pr] = pf_add2(ar[q * 4 + pr], pf_pack2(r[8 * pr + 6], r[8 * pr + 7]));
             }
           }
+          // D is in the accumulators: the issuer may overwrite the buffer while the outputs below are written
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&ctl.d_empty[b]);
           // Blocks that end at this slice are written.  Which of the warpgroup's slots end at (column, t), where
           // their rows sit in the tables and the 1 / n of each block were worked out on the host: the output
           // step is a table look-up and two predicated stores per slot; a group of four slots none of which ends
@@ -390,9 +394,6 @@ k_plan_fused(const __grid_constant__ PlanMaps maps, const __grid_constant__ Shap
               }
             }
           }
-          ptx::tc_fence_before();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(&ctl.d_empty[b]);           // after the outputs: keeps the warps within two slices
         }
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ctl.tab_empty[tb]);          // the table buffer may take the item after next
