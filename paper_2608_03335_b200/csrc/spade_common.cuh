@@ -109,7 +109,8 @@ enum : uint32_t {
   SPADE_ST_TIMEOUT = 1,     // status[0]: a bounded wait gave up; status[1] = where, status[2] = item
 };
 // Status words: [0..2] as above, [4] number of failed index checks of the debug build, [5] site of the first
-// one, [6] the offending value, [8] work-item counter of the attention kernel.
+// one, [6] the offending value, [8] work-item counter of the attention kernel, [9] / [10] tickets by which the last CTA
+// of the scheme-choice / pairing-axis kernel finds out that it is the last (left at zero by that CTA).
 
 // Debug build (-DSPADE_DEBUG): every index taken from a list, a histogram or a table is checked before use.
 // A failed check never traps: it is counted in the status words, the first site and value are kept, and the
