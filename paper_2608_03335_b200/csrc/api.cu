@@ -253,6 +253,8 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
     if (g.BS != 64 && g.BS != 128) { const int bs = g.BS; free(p); return fail(SPADE_ERR_UNSUPPORTED, "candidate %d has %d tokens per block (64 or 128 needed)", c, bs); }
     if (g.bt > 128 || g.bh > 128 || g.bw > 128) { free(p); return fail(SPADE_ERR_UNSUPPORTED, "candidate %d: extent above 128", c); }
     g.nbt = (sh.T + g.bt - 1) / g.bt; g.nbh = (sh.H + g.bh - 1) / g.bh; g.nbw = (sh.W + g.bw - 1) / g.bw;
+    g.mag_w = g.nbw > 1 ? (uint32_t)(0x100000000ull / (unsigned long long)g.nbw) + 1u : 0u;
+    g.mag_hw = g.nbw * g.nbh > 1 ? (uint32_t)(0x100000000ull / ((unsigned long long)g.nbw * g.nbh)) + 1u : 0u;
     g.NBv = g.nbt * g.nbh * g.nbw;
     g.NBt = (sh.n_text + g.BS - 1) / g.BS;
     g.NB = g.NBv + g.NBt;

@@ -113,7 +113,8 @@ __device__ __forceinline__ void load_kv_unit(uint8_t* dst, const CandMaps& vm, c
     ptx::tma_load_3d(dst, tmap, bar, 0, row, bh);
     ptx::tma_load_3d(dst + KSUB_BYTES, tmap, bar, 64, row, bh);
   } else {
-    const int iw = blk % g.nbw, ih = (blk / g.nbw) % g.nbh, it = blk / (g.nbw * g.nbh);
+    int it, ih, iw;
+    block_coords(g, blk, it, ih, iw);          // two high multiplies: this runs per unit in a thread that shares a scheduler with a softmax warp
     const int w0 = iw * g.bw + half * g.hw, h0 = ih * g.bh + half * g.hh, t0 = it * g.bt + half * g.ht;
     ptx::tma_load_5d(dst, vmap, bar, 0, w0, h0, t0, bh);
     ptx::tma_load_5d(dst + KSUB_BYTES, vmap, bar, 64, w0, h0, t0, bh);

@@ -26,8 +26,21 @@ struct CandGeo {
   float inv_z;           // 1 / (2 * sum_i n_i^2): normaliser of the Aggregation Score
   int kt, kh, kw;        // extents of a 64-row K/V box: the block itself (BS 64) or its first half (BS 128)
   int ht, hh, hw;        // origin offset of the second half of a 128-token block (0 for BS 64)
-  int pad;
+  uint32_t mag_w, mag_hw; // floor(2^32 / nbw) + 1 and floor(2^32 / (nbw * nbh)) + 1: block id -> (it, ih, iw) with two high
+                         // multiplies (exact for ids below 2^16) instead of three divisions
 };
+
+// Block id -> block coordinates along (t, h, w), for ids below 2^16.
+__host__ __device__ __forceinline__ void block_coords(const CandGeo& g, int blk, int& it, int& ih, int& iw) {
+#ifdef __CUDA_ARCH__
+  it = g.mag_hw ? (int)__umulhi((unsigned)blk, g.mag_hw) : blk;          // 0 stands for a divisor of 1
+  const int rem = blk - it * (g.nbw * g.nbh);
+  ih = g.mag_w ? (int)__umulhi((unsigned)rem, g.mag_w) : rem;
+  iw = rem - ih * g.nbw;
+#else
+  iw = blk % g.nbw; ih = (blk / g.nbw) % g.nbh; it = blk / (g.nbw * g.nbh);
+#endif
+}
 
 struct Shape {
   int BH, N, Nv, n_text, T, H, W, C;
