@@ -385,6 +385,12 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
       //  doing both products would hold back O += P V of unit j behind the issue of S of unit j+1)
       const uint32_t idesc_s = ptx::idesc_bf16(128, 64, false);
       const uint32_t aQ = ptx::smem_u32(sQ), aK = ptx::smem_u32(sK);
+      // Descriptors differ from a base only in the 16-byte address units of their low bits (shared-memory addresses stay
+      // below 2^18, so nothing carries): the eight of Q are fixed, K's are a base per stage plus a constant per step.
+      uint64_t qd[8];
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) qd[ks] = ptx::smem_desc_sw128(aQ + (ks >> 2) * SUB_BYTES + (ks & 3) * 32, 16, 1024);
+      const uint64_t kd0 = ptx::smem_desc_sw128(aK, 16, 1024);
       uint32_t it = 0, hc = 0;
       for (;; ++it) {
         uint32_t site = 0;
@@ -399,13 +405,10 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
           if (!ptx::mbar_wait(&ctl.k_full[b], u, &ctl.abort, WAIT_NS) ||
               !ptx::mbar_wait(&ctl.s_free, (h & 1) ^ 1, &ctl.abort, WAIT_NS)) { site = 7; break; }   // S of unit h-1 is in registers
           ptx::tc_fence_after();
+          const uint64_t kdb = kd0 + (uint64_t)((b * KV_BYTES) >> 4);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {          // both operands K-major, 16 channels per step
-            const uint32_t qoff = (ks >> 2) * SUB_BYTES + (ks & 3) * 32;
-            const uint32_t koff = b * KV_BYTES + (ks >> 2) * KSUB_BYTES + (ks & 3) * 32;
-            ptx::umma_ss(tmem_S, ptx::smem_desc_sw128(aQ + qoff, 16, 1024),
-                         ptx::smem_desc_sw128(aK + koff, 16, 1024), idesc_s, ks > 0);
-          }
+          for (int ks = 0; ks < 8; ++ks)            // both operands K-major, 16 channels per step
+            ptx::umma_ss(tmem_S, qd[ks], kdb + (uint64_t)(((ks >> 2) * KSUB_BYTES + (ks & 3) * 32) >> 4), idesc_s, ks > 0);
           ptx::umma_commit(&ctl.s_full);
           ptx::umma_commit(&ctl.k_empty[b]);
         }
@@ -420,6 +423,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
       const uint32_t aV = ptx::smem_u32(sV);
       // every 8 x 8 core matrix of the 16 x 16 ones operand is the same 128 bytes: strides 0, no swizzle
       const uint64_t desc_ones = (uint64_t)((ptx::smem_u32(ctl.ones) & 0x3ffffu) >> 4) | ((uint64_t)1 << 46);
+      const uint64_t vd0 = ptx::smem_desc_sw128(aV, KSUB_BYTES, 1024);
       uint32_t it = 0, hc = 0;
       for (;; ++it) {
         uint32_t site = 0;
@@ -432,11 +436,10 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
           if (!ptx::mbar_wait(&ctl.p_full, h & 1, &ctl.abort, WAIT_NS) ||
               !ptx::mbar_wait(&ctl.v_full[b], u, &ctl.abort, WAIT_NS)) { site = 8; break; }
           ptx::tc_fence_after();
+          const uint64_t vdb = vd0 + (uint64_t)((b * KV_BYTES) >> 4);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)            // P from TMEM (bf16 pairs), V MN-major, 16 keys per step
-            ptx::umma_ts(tmem_O, tmem_P + ks * 8,
-                         ptx::smem_desc_sw128(aV + b * KV_BYTES + ks * 2048, KSUB_BYTES, 1024), idesc_o,
-                         (j > 0 || ks > 0) ? 1u : 0u);
+            ptx::umma_ts(tmem_O, tmem_P + ks * 8, vdb + (uint64_t)((ks * 2048) >> 4), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)            // L += P 1: the row sums of the weights as the tensor core sees them
             ptx::umma_ts(tmem_L, tmem_P + ks * 8, desc_ones, idesc_l, (j > 0 || ks > 0) ? 1u : 0u);
