@@ -97,7 +97,8 @@ __device__ __forceinline__ void load_q_block(uint8_t* dst, const CandMaps& vm, c
     ptx::tma_load_3d(dst, &tm.q, bar, 0, row, bh);
     ptx::tma_load_3d(dst + SUB_BYTES, &tm.q, bar, 64, row, bh);
   } else {
-    const int iw = blk % g.nbw, ih = (blk / g.nbw) % g.nbh, it = blk / (g.nbw * g.nbh);
+    int it, ih, iw;
+    block_coords(g, blk, it, ih, iw);
     ptx::tma_load_5d(dst, &vm.q, bar, 0, iw * g.bw, ih * g.bh, it * g.bt, bh);
     ptx::tma_load_5d(dst + SUB_BYTES, &vm.q, bar, 64, iw * g.bw, ih * g.bh, it * g.bt, bh);
   }
@@ -128,7 +129,7 @@ __device__ __forceinline__ void store_o_block(const uint8_t* src, const CandMaps
     ptx::tma_store_3d(&tm.o, src, 0, row, bh);
     ptx::tma_store_3d(&tm.o, src + SUB_BYTES, 64, row, bh);
   } else {
-    const int iw = blk % g.nbw, ih = (blk / g.nbw) % g.nbh, it = blk / (g.nbw * g.nbh);
+    const int iw = blk % g.nbw, ih = (blk / g.nbw) % g.nbh, it = blk / (g.nbw * g.nbh);   // once per item, in a softmax thread: the divisions stay (the multiply form moved the hot loop's registers and cost 14 %)
     ptx::tma_store_5d(&vm.o, src, 0, iw * g.bw, ih * g.bh, it * g.bt, bh);
     ptx::tma_store_5d(&vm.o, src + SUB_BYTES, 64, iw * g.bw, ih * g.bh, it * g.bt, bh);
   }
