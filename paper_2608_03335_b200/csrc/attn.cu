@@ -43,7 +43,8 @@ constexpr int TILE_BYTES = 2 * SUB_BYTES;
 constexpr int KSUB_BYTES = 8192;            // K / V unit: 64 rows x 128 B per 64-channel half
 constexpr int KV_BYTES = 2 * KSUB_BYTES;
 constexpr uint64_t WAIT_NS = 2000000000ull; // bound of every device-side wait
-constexpr uint32_t TMEM_COLS = 256;         // S: columns 0..63, P (bf16 pairs): 64..95, row sums L: 96..111, O: 128..255
+constexpr uint32_t TMEM_COLS = 256;         // S: columns 0..63, P (bf16 pairs): 64..95, row sums L: 96..111, Q channels 0..31: 112..127, O: 128..255
+constexpr int Q_TS_STEPS = 2;                // 16-channel steps of S = Q K^T that take Q from tensor memory (what the 16 spare columns hold)
 constexpr unsigned FULL = 0xffffffffu;
 
 // One work item as the producer warp publishes it to the other roles.  The (merged) list itself lives in
@@ -57,7 +58,7 @@ constexpr int V_STAGES = 2;                 // as the scores of unit j are in re
 
 struct Ctl {
   uint64_t list_full[2], list_empty[2];
-  uint64_t q_full, q_empty;
+  uint64_t q_full, q_empty, qt_full;
   uint64_t k_full[K_STAGES], k_empty[K_STAGES], v_full[V_STAGES], v_empty[V_STAGES], s_full, s_free, p_full, pv_done;
   uint32_t tmem_base;
   volatile uint32_t abort;
@@ -172,6 +173,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
     ptx::mbar_init(&ctl.s_free, 4);             // the four softmax warps hold the scores in registers
     ptx::mbar_init(&ctl.q_full, 1);
     ptx::mbar_init(&ctl.q_empty, 2);          // epilogue thread + MMA issuer
+    ptx::mbar_init(&ctl.qt_full, 4);          // one arrival per softmax warp: the first channels of Q are in tensor memory
     ctl.abort = 0;
     for (int i = 0; i < 64; ++i) ctl.ones[i] = 0x3f80;
     ptx::fence_mbar_init();
@@ -187,6 +189,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
   const uint32_t tmem_S = ctl.tmem_base;
   const uint32_t tmem_P = tmem_S + 64;
   const uint32_t tmem_L = tmem_S + 96;        // 16 equal columns: sum over the keys of the bf16 weights, kept by the tensor core
+  const uint32_t tmem_Q = tmem_S + 112;       // Q channels 0..31 as bf16 pairs (operand A of the first two steps of S)
   const uint32_t tmem_O = tmem_S + 128;
   const int total_items = ws.item_start[sh.BH];
   const int total_text = ws.text_start[sh.BH];
@@ -400,6 +403,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
         const int w = ctl.slot[it & 1].item;
         if (H < 0) break;
         if (!site && !ptx::mbar_wait(&ctl.q_full, it & 1, &ctl.abort, WAIT_NS)) site = 6;
+        if (!site && !ptx::mbar_wait(&ctl.qt_full, it & 1, &ctl.abort, WAIT_NS)) site = 19;
         if (!site) ptx::mbar_arrive(&ctl.q_empty);      // this role has seen the tile; the epilogue frees it
         for (int j = 0; j < H && !site; ++j) {
           const uint32_t h = hc + j, b = h % K_STAGES, u = (h / K_STAGES) & 1;
@@ -408,8 +412,13 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
           ptx::tc_fence_after();
           const uint64_t kdb = kd0 + (uint64_t)((b * KV_BYTES) >> 4);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)            // both operands K-major, 16 channels per step
-            ptx::umma_ss(tmem_S, qd[ks], kdb + (uint64_t)(((ks >> 2) * KSUB_BYTES + (ks & 3) * 32) >> 4), idesc_s, ks > 0);
+          for (int ks = 0; ks < 8; ++ks) {          // both operands K-major, 16 channels per step
+            const uint64_t kd = kdb + (uint64_t)(((ks >> 2) * KSUB_BYTES + (ks & 3) * 32) >> 4);
+            // A product with Q in shared memory reads 6 KB per step and takes 48 clk for 32 clk of arithmetic; with Q in
+            // tensor memory it reads K alone and takes the 32
+            if (ks < Q_TS_STEPS) ptx::umma_ts(tmem_S, tmem_Q + ks * 8, kd, idesc_s, ks > 0);
+            else ptx::umma_ss(tmem_S, qd[ks], kd, idesc_s, ks > 0);
+          }
           ptx::umma_commit(&ctl.s_full);
           ptx::umma_commit(&ctl.k_empty[b]);
         }
@@ -468,6 +477,24 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
       const int H = site ? 0 : sl.H, bh = sl.bh, w = sl.item;
       const CandGeo& g = gp.g[site ? 0 : sl.c];
       const uint64_t* kvalid = st.kvalid + (size_t)g.tab_off * 2;
+      if (!site) {
+        // the row's first 32 channels go to tensor memory (the S products of the previous item are complete: their
+        // last scores have been read)
+        if (!__all_sync(FULL, ptx::mbar_wait(&ctl.q_full, it & 1, &ctl.abort, WAIT_NS))) site = 20;
+        if (!site) {
+          uint32_t qa[16];
+#pragma unroll
+          for (int c16 = 0; c16 < 4; ++c16) {
+            const uint4 v = *reinterpret_cast<const uint4*>(sQ + row * 128 + ((c16 ^ (row & 7)) << 4));
+            qa[c16 * 4 + 0] = v.x; qa[c16 * 4 + 1] = v.y; qa[c16 * 4 + 2] = v.z; qa[c16 * 4 + 3] = v.w;
+          }
+          ptx::tmem_st16(tmem_Q + lane_base, qa);
+          ptx::tmem_wait_st();
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&ctl.qt_full);
+        }
+      }
       float m = -INFINITY;
       // List entries are fetched two units ahead and the valid-key masks one unit ahead, each touched only
       // an iteration after its load was issued, so neither latency sits on the critical path.
