@@ -595,13 +595,16 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
         uint32_t pk[32];
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
+          // a chunk of 32 scores at a time: 16 packed scalings, 32 exponentials, 16 packings (independent work next to every exponential)
+          float x[32];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float x0, x1;
-            unpack2(fma2(pack2(__uint_as_float(sr[ch][2 * i]), __uint_as_float(sr[ch][2 * i + 1])), sc2, nb2), x0, x1);
-            const uint32_t pp = ptx::pack_bf16(ptx::ex2(x0), ptx::ex2(x1));
-            pk[ch * 16 + i] = pp;           // their row sum is taken by the tensor core (L += P 1) from these rounded values
-          }
+          for (int i = 0; i < 16; ++i)
+            unpack2(fma2(pack2(__uint_as_float(sr[ch][2 * i]), __uint_as_float(sr[ch][2 * i + 1])), sc2, nb2), x[2 * i], x[2 * i + 1]);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) x[i] = ptx::ex2(x[i]);
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            pk[ch * 16 + i] = ptx::pack_bf16(x[2 * i], x[2 * i + 1]);    // their row sum is taken by the tensor core (L += P 1) from these rounded values
         }
         // P was last read by the products of unit h - 1 (issued about one softmax ago)
         if (!__all_sync(FULL, ptx::mbar_wait(&ctl.pv_done, (h & 1) ^ 1, &ctl.abort, WAIT_NS))) { site = 14; break; }
