@@ -91,12 +91,14 @@ class ClockSampler:
 
 def executed_units(plan, w):
     """128-row x 64-key units the attention kernel multiplies, from the GPU's own lists: two per listed
-    block for 128-token schemes; for 64-token schemes the merged list of each query-block pair (paired
-    along the head's pairing axis, lone blocks where the count along that axis is odd)."""
+    block for 128-token schemes; for 64-token schemes the merged list of each query tile (two blocks of a
+    2 x 2 x 2 cell of the block grid, paired along the axis the head chose for that cell; lone blocks where
+    a cell is a single block; text blocks pair among themselves)."""
     t = plan.tables()
     scheme = t["scheme"].cpu().tolist()
-    axis = t["pair_axis"].cpu().tolist()
+    cell_axis = t["cell_axis"].long()
     total = 0
+    tables = {}
     for bh, c in enumerate(scheme):
         g = plan.geometry(c)
         nb, nbv = g["NB"], g["NBv"]
@@ -109,11 +111,15 @@ def executed_units(plan, w):
         mask = torch.zeros(nb, nb + 1, dtype=torch.bool, device=idx.device)
         mask.scatter_(1, torch.where(valid, idx, torch.full_like(idx, nb)), True)
         mask = mask[:, :nb]
-        dims = [g["nbt"], g["nbh"], g["nbw"]]
-        vm = mask[:nbv].reshape(*dims, nb).movedim(axis[bh], 0)           # pairing axis first
-        if vm.shape[0] % 2:
-            vm = torch.cat([vm, torch.zeros_like(vm[:1])], 0)
-        total += int((vm[0::2] | vm[1::2]).sum())
+        if c not in tables:
+            tc, pr = plan.pair_table(c)
+            tables[c] = (tc.to(idx.device), pr.to(idx.device))
+        tile_cell, pairs = tables[c]
+        axis = cell_axis[bh][tile_cell]                                   # [tiles]
+        e = pairs.gather(1, axis[:, None])[:, 0]
+        qb0, qb1 = e & 0xffff, e >> 16
+        qb1 = torch.where(qb1 == 0xffff, qb0, qb1)
+        total += int((mask[qb0] | mask[qb1]).sum())
         tm = mask[nbv:]
         if tm.shape[0]:
             if tm.shape[0] % 2:
@@ -365,7 +371,13 @@ def main():
 
     t = plan.tables()
     schemes_chosen = t["group_count"].cpu().tolist()[:len(w.candidates)]
-    pairing_axes = [int((t["pair_axis"] == a).sum()) for a in range(3)]
+    pairing_axes = [0, 0, 0]            # cells of the 64-token heads that pair along t, h, w
+    for bh, c in enumerate(t["scheme"].cpu().tolist()):
+        pt = plan.pair_table(c)
+        if pt is not None:
+            ncell = int(pt[0].max()) + 1
+            for a in range(3):
+                pairing_axes[a] += int((t["cell_axis"][bh, :ncell] == a).sum())
     kernel_launches = plan.launch_count()
 
     # ---- end to end through the host-buffer entry point (it lays the workspace out per head chunk) ----

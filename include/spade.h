@@ -174,19 +174,29 @@ typedef struct {
                                      spade_plan, by decreasing list length per query tile after spade_select */
   int32_t* group_count;           /* [C]             heads per scheme */
   int32_t* item_start;            /* [BH+1]          prefix of attention work items over head_order */
-  int32_t* pair_axis;             /* [BH]            64-token schemes: axis (0 t, 1 h, 2 w) along which query blocks pair into tiles */
+  uint8_t* cell_axis;             /* [BH][cell_ld]   64-token schemes: axis (0 t, 1 h, 2 w) along which the query blocks of a 2 x 2 x 2 cell of
+                                     the block grid pair into 128-row tiles (see spade_get_pair_table) */
   uint32_t* status;               /* [4]             device status words (0 = ok) */
   float*   minmax;                /* [4][BH][128][ld] channel-major max/min summaries of the video blocks, ld = block_scores_ld
                                      (NULL with SPADE_EST_MEAN): plane 0 = q_max (SPADE_EST_DSA2) or (q_max + q_min) / 2
                                      (SPADE_EST_DSA), 1 = q_min, 2 = (k_max + k_min) / 2, 3 = (k_max - k_min) / 2 */
   float*   block_scores;          /* [BH][NBvmax][ld] estimator output S of the chosen scheme, ld = block_scores_ld */
   int32_t  block_scores_ld;
+  int32_t  cell_ld;
 } spade_tables_t;
 int spade_get_tables(const spade_plan_t* plan, void* ws, spade_tables_t* out);
 
 /* Per-candidate geometry as the library sees it: out[0..5] = blocks along T, H, W, video blocks,
  * text blocks, block size. */
 int spade_get_geometry(const spade_plan_t* plan, int32_t cand, int32_t* out6);
+
+/* How the attention stage pairs the 64-token query blocks of candidate `cand` into 128-row tiles (Sec. 3.3: the
+ * kernel's tile is 128 rows).  The block grid is cut into cells of 2 x 2 x 2 blocks (fewer at an odd end); after the
+ * index search every head picks, per cell, the axis along which its blocks pair so that the merged lists are shortest
+ * (cell_axis of spade_tables_t).  For video tile t: tile_cell[t] = its cell; pairs[3 t + a] = qb0 | qb1 << 16 are its
+ * blocks when the cell pairs along axis a (qb1 = 0xffff: a lone block).  Host arrays of the returned length (and three
+ * times it), either may be NULL.  Returns the number of video tiles, 0 for a 128-token candidate, or a negative code. */
+int spade_get_pair_table(const spade_plan_t* plan, int32_t cand, int32_t* tile_cell, uint32_t* pairs);
 
 /* Synchronises `stream` and returns SPADE_OK, SPADE_ERR_DEVICE_TIMEOUT (a bounded wait inside a
  * kernel gave up; the output of that call is invalid) or SPADE_ERR_CUDA. */

@@ -49,8 +49,8 @@ class Tables(C.Structure):
                 ("scheme", C.c_void_p), ("keep", C.c_void_p), ("as_", C.c_void_p), ("score", C.c_void_p),
                 ("sics", C.c_void_p), ("NBvmax", C.c_int32), ("qsum", C.c_void_p), ("ksum", C.c_void_p),
                 ("kv_idx", C.c_void_p), ("kv_cnt", C.c_void_p), ("head_order", C.c_void_p),
-                ("group_count", C.c_void_p), ("item_start", C.c_void_p), ("pair_axis", C.c_void_p), ("status", C.c_void_p),
-                ("minmax", C.c_void_p), ("block_scores", C.c_void_p), ("block_scores_ld", C.c_int32)]
+                ("group_count", C.c_void_p), ("item_start", C.c_void_p), ("cell_axis", C.c_void_p), ("status", C.c_void_p),
+                ("minmax", C.c_void_p), ("block_scores", C.c_void_p), ("block_scores_ld", C.c_int32), ("cell_ld", C.c_int32)]
 
 
 _lib = None
@@ -83,6 +83,7 @@ def lib():
         L.spade_forward_host.argtypes = [vp] * 11 + [ip]
         L.spade_get_tables.argtypes = [vp, vp, C.POINTER(Tables)]
         L.spade_get_geometry.argtypes = [vp, C.c_int32, ip]
+        L.spade_get_pair_table.argtypes = [vp, C.c_int32, ip, C.POINTER(C.c_uint32)]
         L.spade_status.argtypes = [vp, vp, vp]
         L.spade_launch_count.argtypes = [vp]
         L.spade_selftest_bounded_wait.argtypes = [vp, C.c_int32, vp]
@@ -205,6 +206,20 @@ class Plan:
         _check(lib().spade_get_geometry(self.handle, cand, out))
         return dict(nbt=out[0], nbh=out[1], nbw=out[2], NBv=out[3], NBt=out[4], BS=out[5], NB=out[3] + out[4])
 
+    def pair_table(self, cand: int):
+        """Tiles of a 64-token candidate: (tile_cell[tiles], pairs[tiles][3]) as int64 tensors on the host;
+        pairs[t][a] = qb0 | qb1 << 16 when the tile's cell pairs along axis a (qb1 = 0xffff: a lone block).
+        None for a 128-token candidate."""
+        n = int(lib().spade_get_pair_table(self.handle, cand, None, None))
+        if n < 0:
+            _check(n)
+        if n == 0:
+            return None
+        tc = (C.c_int32 * n)()
+        pr = (C.c_uint32 * (3 * n))()
+        _check(min(0, int(lib().spade_get_pair_table(self.handle, cand, tc, pr))))
+        return (torch.tensor(list(tc), dtype=torch.int64), torch.tensor(list(pr), dtype=torch.int64).view(n, 3))
+
     # ---- tables (device views into the workspace) ------------------------------------------
     def tables(self) -> Dict[str, torch.Tensor]:
         t = Tables()
@@ -231,5 +246,5 @@ class Plan:
                     ksum=view(t.ksum, f32, (BH, NB, 128)), kv_idx=view(t.kv_idx, i32, (BH, NB, cap)),
                     kv_cnt=view(t.kv_cnt, i32, (BH, NB)), head_order=view(t.head_order, i32, (BH,)),
                     group_count=view(t.group_count, i32, (8,)), item_start=view(t.item_start, i32, (BH + 1,)),
-                    pair_axis=view(t.pair_axis, i32, (BH,)),
+                    cell_axis=view(t.cell_axis, torch.uint8, (BH, t.cell_ld)),
                     status=view(t.status, i32, (4,)), cap=cap, NBmax=NB)

@@ -46,7 +46,7 @@ struct DeviceGuard {
   CUDA_TRY(guard__.err)
 
 struct WsLayout {
-  size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, ksplit, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, nsum, scores, colkeep, rowfull, pair_axis, pair_union, rowbits, mm, qmid, kdsa, text_start, head_work, att_scratch;
+  size_t status, scheme, keep, pthr, as, score, sics, qsum, ksum, ksplit, kv_idx, kv_cnt, head_order, group_count, item_start, cells, csum, nsum, scores, colkeep, rowfull, cell_axis, pair_union, rowbits, mm, qmid, kdsa, text_start, head_work, att_scratch;
   size_t bytes;
   size_t canary[40];     // debug build: offsets of the 256-byte guard words after each region
   int n_canary;
@@ -61,7 +61,9 @@ struct spade_plan_s {
   Shape sh;
   GeoPack gp;
   StaticTables st;
-  void* d_static;        // one allocation holding rowoff, nvalid, kvalid, budget
+  void* d_static;        // one allocation holding rowoff, nvalid, kvalid, budget and the tile tables of the pair schemes
+  uint32_t* h_pair_tab;  // host copies of those tile tables (spade_get_pair_table)
+  int* h_tile_cell;
   WsLayout lay;
   PlanFusedCfg pf;       // one-pass scheme generation (plan.cu), when the candidate set fits it
   PlanMaps* pmaps;       // its tensor maps for the last (Q, K) seen
@@ -111,7 +113,7 @@ WsTables tables_at(const spade_plan_s* p, void* ws) {
   t.csum = (float*)(b + l.csum);
   t.nsum = (float*)(b + l.nsum);
   t.scores = (float*)(b + l.scores);
-  t.pair_axis = (int*)(b + l.pair_axis);
+  t.cell_axis = (uint8_t*)(b + l.cell_axis);
   t.pair_union = (int*)(b + l.pair_union);
   t.rowbits = (uint32_t*)(b + l.rowbits);
   t.colkeep = (uint8_t*)(b + l.colkeep);
@@ -165,7 +167,7 @@ void compute_layout(spade_plan_s* p) {
   l.item_start = take((size_t)(BH + 1) * 4);
   l.text_start = take((size_t)(BH + 1) * 4);
   l.kv_cnt = take((size_t)BH * sh.NBmax * 4);
-  l.pair_axis = take((size_t)BH * 4);
+  l.cell_axis = take((size_t)BH * sh.cell_ld);
   l.pair_union = take((size_t)BH * 4 * 4);
   l.colkeep = take((size_t)BH * sh.NBmax);
   l.rowfull = take((size_t)BH * sh.NBmax);
@@ -260,12 +262,9 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
     g.NB = g.NBv + g.NBt;
     if (g.NB > SPADE_MAX_NB) { const int nb = g.NB; free(p); return fail(SPADE_ERR_UNSUPPORTED, "candidate %d gives %d blocks per head (max %d)", c, nb, SPADE_MAX_NB); }
     g.pair = g.BS == 64;
-    g.vtiles[0] = (g.nbt + 1) / 2 * g.nbh * g.nbw;
-    g.vtiles[1] = g.nbt * ((g.nbh + 1) / 2) * g.nbw;
-    g.vtiles[2] = g.nbt * g.nbh * ((g.nbw + 1) / 2);
     g.ttiles = (g.NBt + 1) / 2;
-    g.tiles = g.NB;
-    if (g.pair) { g.tiles = 0; for (int a = 0; a < 3; ++a) if (g.vtiles[a] + g.ttiles > g.tiles) g.tiles = g.vtiles[a] + g.ttiles; }
+    g.tiles = g.NB;              // pair schemes: set with the tile tables below
+    g.ctiles = 0; g.ncell = 0; g.pt_off = 0; g.pc_off = 0;
     // K/V travel in 64-row boxes: a 128-token block is split along its outermost extended axis
     g.kt = g.bt; g.kh = g.bh; g.kw = g.bw; g.ht = g.hh = g.hw = 0;
     if (!g.pair) {
@@ -333,6 +332,57 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
     g.inv_z = (float)(1.0 / (2.0 * z));
   }
 
+  // Tile tables of the 64-token schemes.  The block grid is cut into cells of 2 x 2 x 2 blocks (fewer at an odd end); the
+  // blocks of a cell are paired along one axis, chosen per head and cell after the index search.  A cell's tiles are the
+  // blocks with offset 0 along that axis, in raster order; an axis along which the cell is one block wide stands for the
+  // first one along which it is two (a cell of one block is a lone tile), so every choice gives the same number of tiles.
+  std::vector<uint32_t> pair_tab;
+  std::vector<int> tile_cell, cell_tile0;
+  sh.cell_ld = 16;
+  for (int c = 0; c < n_cands; ++c) {
+    CandGeo& g = p->gp.g[c];
+    if (!g.pair) continue;
+    g.pt_off = (int)tile_cell.size();
+    g.pc_off = (int)cell_tile0.size();
+    const int nb[3] = {g.nbt, g.nbh, g.nbw}, stride[3] = {g.nbh * g.nbw, g.nbw, 1};
+    const int nc[3] = {(g.nbt + 1) / 2, (g.nbh + 1) / 2, (g.nbw + 1) / 2};
+    g.ncell = nc[0] * nc[1] * nc[2];
+    int tiles = 0;
+    for (int cell = 0; cell < g.ncell; ++cell) {
+      const int cc[3] = {cell / (nc[1] * nc[2]), (cell / nc[2]) % nc[1], cell % nc[2]};
+      int ext[3], first_wide = -1;
+      for (int a = 0; a < 3; ++a) {
+        ext[a] = nb[a] - 2 * cc[a] >= 2 ? 2 : 1;
+        if (ext[a] == 2 && first_wide < 0) first_wide = a;
+      }
+      cell_tile0.push_back(tiles);
+      const int origin = 2 * cc[0] * stride[0] + 2 * cc[1] * stride[1] + 2 * cc[2] * stride[2];
+      const int ntile = first_wide < 0 ? 1 : ext[0] * ext[1] * ext[2] / 2;
+      const size_t at = pair_tab.size();
+      pair_tab.resize(at + (size_t)ntile * 3);
+      for (int a = 0; a < 3; ++a) {
+        const int ax = first_wide < 0 ? -1 : (ext[a] == 2 ? a : first_wide);
+        int k = 0;
+        for (int o0 = 0; o0 < ext[0]; ++o0)
+          for (int o1 = 0; o1 < ext[1]; ++o1)
+            for (int o2 = 0; o2 < ext[2]; ++o2) {
+              const int off[3] = {o0, o1, o2};
+              if (ax >= 0 && off[ax] != 0) continue;
+              const int qb0 = origin + o0 * stride[0] + o1 * stride[1] + o2 * stride[2];
+              const uint32_t qb1 = ax >= 0 ? (uint32_t)(qb0 + stride[ax]) : 0xffffu;
+              pair_tab[at + (size_t)k * 3 + a] = (uint32_t)qb0 | (qb1 << 16);
+              ++k;
+            }
+      }
+      for (int k = 0; k < ntile; ++k) tile_cell.push_back(cell);
+      tiles += ntile;
+    }
+    cell_tile0.push_back(tiles);
+    g.ctiles = tiles;
+    g.tiles = g.ctiles + g.ttiles;
+    if (((g.ncell + 15) & ~15) > sh.cell_ld) sh.cell_ld = (g.ncell + 15) & ~15;
+  }
+
   cudaError_t e = cudaSetDevice(device);
   cudaDeviceProp prop;
   if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, device);
@@ -344,7 +394,10 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
   const size_t o_nvalid = align_up(o_rowoff + rowoff.size() * 4, 256);
   const size_t o_kvalid = align_up(o_nvalid + nvalid.size() * 4, 256);
   const size_t o_budget = align_up(o_kvalid + kvalid.size() * 8, 256);
-  const size_t total = align_up(o_budget + bud.size() * 4, 256);
+  const size_t o_ptab = align_up(o_budget + bud.size() * 4, 256);
+  const size_t o_tcell = align_up(o_ptab + pair_tab.size() * 4, 256);
+  const size_t o_ctile = align_up(o_tcell + tile_cell.size() * 4, 256);
+  const size_t total = align_up(o_ctile + cell_tile0.size() * 4, 256);
   e = cudaMalloc(&p->d_static, total);
   if (e != cudaSuccess) { free(p); return fail(SPADE_ERR_CUDA, "cudaMalloc(%zu): %s", total, cudaGetErrorString(e)); }
   char* base = (char*)p->d_static;
@@ -352,11 +405,17 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
   if (e == cudaSuccess) e = cudaMemcpy(base + o_nvalid, nvalid.data(), nvalid.size() * 4, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemcpy(base + o_kvalid, kvalid.data(), kvalid.size() * 8, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemcpy(base + o_budget, bud.data(), bud.size() * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && !pair_tab.empty()) e = cudaMemcpy(base + o_ptab, pair_tab.data(), pair_tab.size() * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && !tile_cell.empty()) e = cudaMemcpy(base + o_tcell, tile_cell.data(), tile_cell.size() * 4, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && !cell_tile0.empty()) e = cudaMemcpy(base + o_ctile, cell_tile0.data(), cell_tile0.size() * 4, cudaMemcpyHostToDevice);
   if (e != cudaSuccess) { cudaFree(p->d_static); free(p); return fail(SPADE_ERR_CUDA, "table upload: %s", cudaGetErrorString(e)); }
   p->st.rowoff = (const uint32_t*)(base + o_rowoff);
   p->st.nvalid = (const int*)(base + o_nvalid);
   p->st.kvalid = (const uint64_t*)(base + o_kvalid);
   p->st.budget = (const float*)(base + o_budget);
+  p->st.pair_tab = (const uint32_t*)(base + o_ptab);
+  p->st.tile_cell = (const int*)(base + o_tcell);
+  p->st.cell_tile0 = (const int*)(base + o_ctile);
 
   p->base_cap = sh.cap;
   plan_fused_configure(&p->pf, sh, p->gp, p->num_sms);
@@ -377,10 +436,14 @@ int spade_plan_create(spade_plan_t** out, int32_t B, int32_t heads, int32_t d, c
   p->maps = (AttnMaps*)calloc(1, attn_maps_bytes());
   p->smaps = (ScoreMaps*)calloc(1, score_maps_bytes());
   p->pmaps = (PlanMaps*)calloc(1, plan_maps_bytes());
-  if (!p->maps || !p->smaps || !p->pmaps) {
-    cudaFree(p->d_static); free(p->maps); free(p->smaps); free(p->pmaps); free(p);
+  p->h_pair_tab = (uint32_t*)malloc(pair_tab.size() * 4 + 4);
+  p->h_tile_cell = (int*)malloc(tile_cell.size() * 4 + 4);
+  if (!p->maps || !p->smaps || !p->pmaps || !p->h_pair_tab || !p->h_tile_cell) {
+    cudaFree(p->d_pf); cudaFree(p->d_static); free(p->maps); free(p->smaps); free(p->pmaps); free(p->h_pair_tab); free(p->h_tile_cell); free(p);
     return fail(SPADE_ERR_INVALID_ARG, "out of host memory");
   }
+  if (!pair_tab.empty()) memcpy(p->h_pair_tab, pair_tab.data(), pair_tab.size() * 4);
+  if (!tile_cell.empty()) memcpy(p->h_tile_cell, tile_cell.data(), tile_cell.size() * 4);
   *out = p;
   return SPADE_OK;
 }
@@ -398,6 +461,8 @@ int spade_plan_destroy(spade_plan_t* p) {
   free(p->maps);
   free(p->smaps);
   free(p->pmaps);
+  free(p->h_pair_tab);
+  free(p->h_tile_cell);
   free(p);
   return SPADE_OK;
 }
@@ -439,6 +504,16 @@ int spade_get_geometry(const spade_plan_t* p, int32_t c, int32_t* out6) {
   return SPADE_OK;
 }
 
+int spade_get_pair_table(const spade_plan_t* p, int32_t c, int32_t* tile_cell, uint32_t* pairs) {
+  if (!p) return fail(SPADE_ERR_INVALID_ARG, "plan is NULL");
+  if (c < 0 || c >= p->sh.C) return fail(SPADE_ERR_INVALID_ARG, "candidate %d out of range", c);
+  const CandGeo& g = p->gp.g[c];
+  if (!g.pair) return 0;
+  if (tile_cell) memcpy(tile_cell, p->h_tile_cell + g.pt_off, (size_t)g.ctiles * 4);
+  if (pairs) memcpy(pairs, p->h_pair_tab + (size_t)g.pt_off * 3, (size_t)g.ctiles * 3 * 4);
+  return g.ctiles;
+}
+
 int spade_get_tables(const spade_plan_t* p, void* ws, spade_tables_t* out) {
   int rc = check_call(p, ws);
   if (rc) return rc;
@@ -449,7 +524,8 @@ int spade_get_tables(const spade_plan_t* p, void* ws, spade_tables_t* out) {
   out->NBvmax = p->sh.NBvmax;
   out->qsum = t.qsum; out->ksum = t.ksum; out->kv_idx = t.kv_idx; out->kv_cnt = t.kv_cnt;
   out->head_order = t.head_order; out->group_count = t.group_count; out->item_start = t.item_start;
-  out->pair_axis = t.pair_axis;
+  out->cell_axis = t.cell_axis;
+  out->cell_ld = p->sh.cell_ld;
   out->status = t.status;
   out->minmax = p->sh.estimator ? t.mm : nullptr;
   out->block_scores = t.scores;
@@ -569,7 +645,7 @@ int spade_select(spade_plan_t* p, void* ws, void* stream) {
   if (any_pair) {
     // pair the 64-token query blocks along the axis that gives the shortest merged lists, per head (the totals start
     // at zero: the plan stage and the previous use leave them so); the kernel's last CTA then orders the heads
-    CUDA_TRY(launch_pair_axis(p->sh, p->gp, t, p->num_sms, (cudaStream_t)stream));
+    CUDA_TRY(launch_pair_axis(p->sh, p->gp, p->st, t, p->num_sms, (cudaStream_t)stream));
   } else {
     CUDA_TRY(launch_groups_after_select(p->sh, p->gp, t, (cudaStream_t)stream));
   }

@@ -44,6 +44,9 @@ constexpr int KSUB_BYTES = 8192;            // K / V unit: 64 rows x 128 B per 6
 constexpr int KV_BYTES = 2 * KSUB_BYTES;
 constexpr uint64_t WAIT_NS = 2000000000ull; // bound of every device-side wait
 constexpr uint32_t TMEM_COLS = 256;         // S: columns 0..63, P (bf16 pairs): 64..95, row sums L: 96..111, Q channels 0..31: 112..127, O: 128..255
+#ifndef ATT_CODE_PAD
+#define ATT_CODE_PAD 256    // instructions; see the softmax role.  Attention time repeats with a period of 512 (8 KB): fastest at 192..320
+#endif
 constexpr int Q_TS_STEPS = 2;                // 16-channel steps of S = Q K^T that take Q from tensor memory (what the 16 spare columns hold)
 constexpr unsigned FULL = 0xffffffffu;
 
@@ -259,7 +262,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
         const int n_video_tiles = v_hi - v_lo;
         const int tile = text_item ? n_video_tiles + (wi - t_lo) : wi - v_lo;
         int qb0, qb1;
-        tile_blocks(g, ws.pair_axis[bh], tile, qb0, qb1);
+        tile_blocks(g, st, ws.cell_axis + (size_t)bh * sh.cell_ld, tile, qb0, qb1);
         int n_entries;
         if (g.pair) {
           // merged (union) list of the two 64-token query blocks, via a bitmap over KV block ids
@@ -464,6 +467,15 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
   } else {
     // ================= softmax + epilogue (warps 0..3, one query row per thread) ======================
     reg_inc<REGS_SOFTMAX>();
+    // Never taken (BH is positive).  The instructions it keeps in the binary shift the loop below against the loops of the
+    // helper roles in the instruction cache.  Measured over paddings of 0..2048 instructions: attention time repeats every
+    // 512 instructions (8 KB), 2.02-2.04 ms at 0, 512, 1024, ... and 1.80 ms at 192..320 and 768 on the Wan-1.3B shape, with
+    // the same instructions executed and instruction-fetch stalls per issue of 1.5 against 0.7: the loops evict one another
+    // when they fall on the same cache sets.
+    if (sh.BH < 0) {
+#pragma unroll
+      for (int i = 0; i < ATT_CODE_PAD; ++i) asm volatile("nanosleep.u32 1;");
+    }
     const int row = warp * 32 + lane;
     const int qhalf = row >> 6;
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
@@ -521,7 +533,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
         const bool all_valid = __all_sync(FULL, mask == ~0ull);
         if (!__all_sync(FULL, ptx::mbar_wait(&ctl.s_full, h & 1, &ctl.abort, WAIT_NS))) { site = 10; break; }
         ptx::tc_fence_after();
-        if (__all_sync(FULL, mask == 0ull)) {
+        if (__builtin_expect(__all_sync(FULL, mask == 0ull), 0)) {
           // None of this warp's 32 rows takes part in the unit (the other half of a paired tile listed it, or the
           // unit holds no real key): its weights are exact zeros, no score is read and no exponential is taken.
           ptx::tc_fence_before();
@@ -546,7 +558,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
         ptx::tc_fence_before();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&ctl.s_free);      // the scores are in registers: S of the next unit may be issued
-        if (!all_valid) {
+        if (__builtin_expect(!all_valid, 0)) {
 #pragma unroll
           for (int ch = 0; ch < 2; ++ch) {
             const uint32_t bits = (uint32_t)(mask >> (ch * 32));
@@ -564,7 +576,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
         const float m_new = max3(m, mxa, mxb);
         // lazy rescale: move the reference maximum only when it grew by more than 2^8
         const bool grow = (m_new - m) * scale_log2 > 8.f;     // also true the first time a finite score appears
-        if (__any_sync(FULL, grow)) {
+        if (__builtin_expect(__any_sync(FULL, grow), 0)) {      // rare: laid out away from the loop, like the other unlikely branches
           if (j > 0) {
             const uint32_t hp = h - 1;                          // O must hold every product issued so far
             if (!__all_sync(FULL, ptx::mbar_wait(&ctl.pv_done, hp & 1, &ctl.abort, WAIT_NS))) { site = 11; break; }

@@ -389,10 +389,9 @@ k_choose(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, S
 // Order in which the attention kernel takes the heads, heads per scheme, and the prefixes of attention
 // work items (all query tiles, and the text query tiles alone: those attend every block and are handed
 // out first).
-// mode 0 (plan stage, lists unknown): heads grouped by scheme (Sec. 3.3), pairing axis reset to w.
+// mode 0 (plan stage, lists unknown): heads grouped by scheme (Sec. 3.3), every cell's pairing axis reset to w.
 // mode 1 (after the index search): heads by decreasing list length per query tile, so that the longest
-// work items start first and the last ones are short; pairing axis = argmin of the merged-list totals
-// that k_pair_axis measured (ties -> w, then h, then t).
+// work items start first and the last ones are short (k_pair_axis has set the cells' axes).
 // Runs in ONE CTA (every thread of it): k_groups, or the last CTA to finish of k_choose (mode 0) / k_pair_axis (mode 1).
 __device__ __forceinline__ void groups_body(const Shape& sh, const GeoPack& gp, const WsTables& ws, int mode) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -423,16 +422,9 @@ __device__ __forceinline__ void groups_body(const Shape& sh, const GeoPack& gp, 
       // 64-token query blocks is somewhat shorter than both lists together
       key = (float)sum / (float)g.NBv * (g.pair ? 1.7f : 2.0f);
     }
-    if (lane == 0) {
-      int axis = 2;
-      if (mode == 1 && g.pair) {
-        const int u0 = __ldcg(ws.pair_union + bh * 4), u1 = __ldcg(ws.pair_union + bh * 4 + 1), u2 = __ldcg(ws.pair_union + bh * 4 + 2);
-        if (u1 < u2) axis = 1;
-        if (u0 < (axis == 1 ? u1 : u2)) axis = 0;
-      }
-      ws.pair_axis[bh] = axis;
-      ws.head_work[bh] = key;
-    }
+    if (mode == 0 && g.pair)
+      for (int i = lane; i < sh.cell_ld; i += 32) ws.cell_axis[(size_t)bh * sh.cell_ld + i] = 2;
+    if (lane == 0) ws.head_work[bh] = key;
   }
   __syncthreads();
   for (int i = tid; i < sh.BH; i += nthreads) {                  // rank = heads that come before head i
@@ -444,7 +436,7 @@ __device__ __forceinline__ void groups_body(const Shape& sh, const GeoPack& gp, 
     }
     const int c = __ldcg(ws.scheme + i);
     ws.head_order[rank] = i;
-    ws.item_start[rank + 1] = head_tiles(gp.g[c], ws.pair_axis[i]);      // counts; scanned below
+    ws.item_start[rank + 1] = head_tiles(gp.g[c]);      // counts; scanned below
     ws.text_start[rank + 1] = gp.g[c].pair ? gp.g[c].ttiles : gp.g[c].NBt;
     atomicAdd(&ws.group_count[c], 1);
   }
@@ -490,39 +482,47 @@ __device__ __forceinline__ bool last_cta_done(uint32_t* status, int word) {
   return last_sm != 0;
 }
 
-// Merged-list length of a head's query tiles for each pairing axis (on a sample of the blocks): one warp
-// per (head, axis, sampled video block with an even coordinate along the axis) adds |L_i u L_j| of the pair (or |L_i| of a lone
-// block), read off the bitmaps of the lists that the index search leaves next to them.
+// Pairing axis of every cell of a head's block grid (64-token schemes): one warp per (head, cell) adds up, for each of the
+// three axes, the merged-list lengths |L_i u L_j| of the cell's tiles (|L_i| of a lone block) -- popcounts over the bitmaps
+// the index search leaves next to the lists; the text blocks every list ends with do not change the ranking -- and keeps
+// the axis with the smallest total (ties -> w, then h, then t).
 __global__ void __launch_bounds__(WARPS_PER_CTA * 32)
-k_pair_axis(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, WsTables ws) {
+k_pair_axis(const __grid_constant__ Shape sh, const __grid_constant__ GeoPack gp, StaticTables st, WsTables ws) {
   const int lane = threadIdx.x & 31;
   const int gw = blockIdx.x * WARPS_PER_CTA + (threadIdx.x >> 5);
   const int nw = gridDim.x * WARPS_PER_CTA;
-  const int total = sh.BH * 3 * sh.NBvmax;            // at most 4096 * 3 * 2048
+  const int total = sh.BH * sh.cell_ld;               // at most 4096 * 2048
   for (int u = gw; u < total; u += nw) {
-    const int i = u % sh.NBvmax, axis = (u / sh.NBvmax) % 3, bh = u / (3 * sh.NBvmax);
+    const int cell = u % sh.cell_ld, bh = u / sh.cell_ld;
     const CandGeo& g = gp.g[ws.scheme[bh]];
-    if (!g.pair || i >= g.NBv) continue;
-    // a deterministic sample of about 400 blocks per head is enough to rank the three axes
-    const uint32_t stride = (uint32_t)(g.NBv / 400) + 1u;
-    if (((uint32_t)i * 2654435761u >> 12) % stride != 0u) continue;
-    const int cw = i % g.nbw, chh = (i / g.nbw) % g.nbh, ct = i / (g.nbw * g.nbh);
-    const int ca = axis == 2 ? cw : axis == 1 ? chh : ct;
-    const int na = axis == 2 ? g.nbw : axis == 1 ? g.nbh : g.nbt;
-    if (ca & 1) continue;
-    // |L_i u L_j| over the video KV blocks = popcount of the OR of the two rows' bitmaps (the text blocks every
-    // list ends with are the same for all rows and do not change the ranking of the axes)
-    const uint32_t* Bi = ws.rowbits + ((size_t)bh * sh.NBvmax + i) * sh.bits_ld;
+    if (!g.pair || cell >= g.ncell) continue;
+    const int t0 = __ldg(st.cell_tile0 + g.pc_off + cell), t1 = __ldg(st.cell_tile0 + g.pc_off + cell + 1);
+    const uint32_t* rows = ws.rowbits + (size_t)bh * sh.NBvmax * sh.bits_ld;
     const int words = (g.NBv + 31) >> 5;
-    const uint32_t* Bj = Bi;
-    if (ca + 1 < na) Bj = Bi + (size_t)(axis == 2 ? 1 : axis == 1 ? g.nbw : g.nbw * g.nbh) * sh.bits_ld;
-    int uni = 0;
-    for (int wd = lane; wd < words; wd += 32) uni += __popc(Bi[wd] | Bj[wd]);
+    int cost[3] = {0, 0, 0};
+    for (int t = t0; t < t1; ++t) {
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) uni += __shfl_xor_sync(FULL, uni, o);
-    if (lane == 0) atomicAdd(&ws.pair_union[bh * 4 + axis], uni);
+      for (int a = 0; a < 3; ++a) {
+        const uint32_t e = __ldg(st.pair_tab + (size_t)(g.pt_off + t) * 3 + a);
+        const uint32_t qb0 = e & 0xffffu, qb1 = (e >> 16) == 0xffffu ? qb0 : (e >> 16);
+        if (!SPADE_CHECK(qb0 < (uint32_t)g.NBv && qb1 < (uint32_t)g.NBv, ws.status, 501, (int)e)) continue;
+        const uint32_t* Bi = rows + (size_t)qb0 * sh.bits_ld;
+        const uint32_t* Bj = rows + (size_t)qb1 * sh.bits_ld;
+        for (int wd = lane; wd < words; wd += 32) cost[a] += __popc(Bi[wd] | Bj[wd]);
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < 3; ++a)
+#pragma unroll
+      for (int o = 16; o >= 1; o >>= 1) cost[a] += __shfl_xor_sync(FULL, cost[a], o);
+    if (lane == 0) {
+      int axis = 2;
+      if (cost[1] < cost[2]) axis = 1;
+      if (cost[0] < cost[axis]) axis = 0;
+      ws.cell_axis[(size_t)bh * sh.cell_ld + cell] = (uint8_t)axis;
+    }
   }
-  // the last CTA to get here picks the axes and orders the heads by list length
+  // the last CTA to get here orders the heads by list length
   if (last_cta_done(ws.status, 10)) groups_body(sh, gp, ws, 1);
 }
 
@@ -1224,11 +1224,11 @@ cudaError_t launch_groups_after_select(const Shape& sh, const GeoPack& gp, const
   return cudaGetLastError();
 }
 
-cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s) {
-  const long total = (long)sh.BH * 3 * sh.NBvmax;
+cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws, int num_sms, cudaStream_t s) {
+  const long total = (long)sh.BH * sh.cell_ld;
   long ctas = (total + WARPS_PER_CTA - 1) / WARPS_PER_CTA;
   if (ctas > (long)num_sms * 8) ctas = (long)num_sms * 8;
-  k_pair_axis<<<(unsigned)ctas, WARPS_PER_CTA * 32, 0, s>>>(sh, gp, ws);
+  k_pair_axis<<<(unsigned)ctas, WARPS_PER_CTA * 32, 0, s>>>(sh, gp, st, ws);
   return cudaGetLastError();
 }
 

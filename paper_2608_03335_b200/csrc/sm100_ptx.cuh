@@ -45,7 +45,7 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
 // SM cycle counter is read only every 256 failed polls (the clock is at most ~2 GHz, so
 // limit_ns * 2 cycles is a safe upper bound of the limit).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort, uint64_t limit_ns) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (__builtin_expect(mbar_try_wait(bar, parity), 1)) return true;         // (the polling loop is laid out away from the callers' hot loops)
   uint32_t spins = 0;
   long long t0 = 0;
   for (;;) {

@@ -19,7 +19,9 @@ struct CandGeo {
   int NBv, NBt, NB, BS;  // video blocks, text blocks, total, nominal block size (64 or 128)
   int pair;              // 1 when BS == 64: two consecutive query blocks share one 128-row tile
   int tiles;             // upper bound of attention work items per head
-  int vtiles[3];         // pair schemes: video query tiles when blocks are paired along t, h or w
+  int ctiles;            // pair schemes: video query tiles (blocks are paired inside 2 x 2 x 2 cells of the block grid, along an axis chosen per cell)
+  int ncell;             // pair schemes: cells of the block grid = ceil(nbt/2) * ceil(nbh/2) * ceil(nbw/2)
+  int pt_off, pc_off;    // pair schemes: offsets of this candidate's rows in the tile tables (pair_tab, tile_cell) and in cell_tile0
   int ttiles;            // pair schemes: text query tiles = ceil(NBt / 2)
   int unit_off;          // prefix of NBv over candidates (unit decoding of the SICS pass)
   int tab_off;           // offset of this candidate's rows in the per-block tables (nvalid, kvalid)
@@ -59,6 +61,7 @@ struct Shape {
   int CS;                   // tokens per full cell
   int ld_scores;            // row length of the block-score scratch (NBvmax rounded up to 64)
   int bits_ld;              // 32-bit words per row of the list bitmaps (ld_scores / 32)
+  int cell_ld;              // bytes per head of the cell-axis table (largest cell count over the pair candidates, rounded up to 16)
   // static / intra-block masks united with the dynamic selection (masks_on = any of them enabled)
   int masks_on, window, sink;
   float intra_thr;
@@ -71,6 +74,11 @@ struct StaticTables {
   const int* nvalid;        // [sum NB_c] valid tokens per block
   const uint64_t* kvalid;   // [sum NB_c][2] bit r set <=> in-block row r is a real token
   const float* budget;      // [BH] per-head budget value (k, p or sparsity)
+  // pair schemes (64-token blocks): the video tiles of a cell are consecutive; a tile's two blocks depend on the cell's axis
+  const uint32_t* pair_tab; // [sum ctiles][3] tile, axis (0 t, 1 h, 2 w) -> qb0 | qb1 << 16 (0xffff: lone block); an axis along which the
+                            // cell is one block wide repeats the entry of one that is not
+  const int* tile_cell;     // [sum ctiles] tile -> cell
+  const int* cell_tile0;    // [sum (ncell + 1)] cell -> its first tile
 };
 
 // Pointers into the caller's workspace.
@@ -95,7 +103,7 @@ struct WsTables {
   float* cells;         // [BH][2 tensors][NCELL][2 (sum of q/|q|, sum of q)][128]
   float* csum;          // [BH][2 tensors][C][NBmax][128] mean summaries of every candidate
   float* nsum;          // same shape: sum over a block's tokens of q / |q| (one-pass scheme generation only)
-  int* pair_axis;       // [BH] axis (0 t, 1 h, 2 w) along which 64-token query blocks are paired into 128-row tiles
+  uint8_t* cell_axis;   // [BH][cell_ld] axis (0 t, 1 h, 2 w) along which the 64-token query blocks of a cell are paired into 128-row tiles
   int* pair_union;      // [BH][4] total merged-list length for each pairing axis; [3] = blocks listed over the head's video query rows
   uint32_t* rowbits;    // [BH][NBvmax][bits_ld] the video part of every video query block's list as a bitmap (bit j = KV block j kept)
   uint8_t* colkeep;     // [BH][NBmax] KV block kept by every query block (intra rule on K, sink)
@@ -172,7 +180,7 @@ cudaError_t launch_gather(const Shape& sh, const GeoPack& gp, const WsTables& ws
 cudaError_t launch_split_k(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_choose(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws,
                           const ForcedPack& forced, int have_sics, cudaStream_t s);
-cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const WsTables& ws, int num_sms, cudaStream_t s);
+cudaError_t launch_pair_axis(const Shape& sh, const GeoPack& gp, const StaticTables& st, const WsTables& ws, int num_sms, cudaStream_t s);
 cudaError_t launch_groups_after_select(const Shape& sh, const GeoPack& gp, const WsTables& ws, cudaStream_t s);
 cudaError_t launch_summarize(const void* Q, const void* K, const Shape& sh, const GeoPack& gp, const StaticTables& st,
                              const WsTables& ws, int num_sms, cudaStream_t s);
@@ -209,28 +217,23 @@ cudaError_t launch_selftest_wait(uint32_t* out, unsigned long long limit_ns, cud
 int attn_encode_maps(AttnMaps* out, const void* Q, const void* K, const void* V, void* O, const Shape& sh,
                      const GeoPack& gp, char* err, size_t errlen);
 
-// Query tile -> its one or two query blocks.  128-token schemes: the block itself.  64-token schemes:
-// two blocks adjacent along `axis` (0 t, 1 h, 2 w) starting at an even coordinate (a lone block when
-// the count along that axis is odd); text blocks are paired among themselves after the video tiles.
-__host__ __device__ inline void tile_blocks(const CandGeo& g, int axis, int tile, int& qb0, int& qb1) {
+// Query tile -> its one or two query blocks.  128-token schemes: the block itself.  64-token schemes: two blocks of one
+// 2 x 2 x 2 cell of the block grid, adjacent along the cell's axis (a lone block where the cell is a single block); text
+// blocks are paired among themselves after the video tiles.
+__device__ __forceinline__ void tile_blocks(const CandGeo& g, const StaticTables& st, const uint8_t* cell_axis, int tile, int& qb0, int& qb1) {
   if (!g.pair) { qb0 = tile; qb1 = -1; return; }
-  const int vt = g.vtiles[axis];
-  if (tile >= vt) {
-    qb0 = g.NBv + 2 * (tile - vt);
+  if (tile >= g.ctiles) {
+    qb0 = g.NBv + 2 * (tile - g.ctiles);
     qb1 = qb0 + 1 < g.NB ? qb0 + 1 : -1;
     return;
   }
-  int n[3] = {g.nbt, g.nbh, g.nbw};
-  const int na = n[axis];
-  n[axis] = (na + 1) >> 1;
-  int c[3];
-  c[2] = tile % n[2]; c[1] = (tile / n[2]) % n[1]; c[0] = tile / (n[2] * n[1]);
-  c[axis] *= 2;
-  qb0 = (c[0] * g.nbh + c[1]) * g.nbw + c[2];
-  const int stride = axis == 2 ? 1 : axis == 1 ? g.nbw : g.nbw * g.nbh;
-  qb1 = c[axis] + 1 < na ? qb0 + stride : -1;
+  int axis = cell_axis[__ldg(st.tile_cell + g.pt_off + tile)];
+  axis = axis > 2 ? 2 : axis;
+  const uint32_t e = __ldg(st.pair_tab + (size_t)(g.pt_off + tile) * 3 + axis);
+  qb0 = (int)(e & 0xffffu);
+  qb1 = (e >> 16) == 0xffffu ? -1 : (int)(e >> 16);
 }
-__host__ __device__ inline int head_tiles(const CandGeo& g, int axis) { return g.pair ? g.vtiles[axis] + g.ttiles : g.NB; }
+__host__ __device__ inline int head_tiles(const CandGeo& g) { return g.pair ? g.ctiles + g.ttiles : g.NB; }
 
 __device__ __forceinline__ void bf16x8_to_float(const uint4& v, float* x) {
   x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);

@@ -596,3 +596,36 @@ def test_topp_lists_are_reproducible_bit_for_bit_also_through_a_graph():
         plan.spade_status()
     finally:
         plan.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("grid,cand", [((21, 45, 80), (8, 2, 4)), ((21, 45, 80), (4, 4, 4)), ((16, 45, 80), (16, 1, 4)),
+                                       ((5, 7, 9), (1, 1, 64)), ((1, 8, 8), (1, 8, 8)), ((3, 3, 3), (4, 4, 4))])
+def test_tile_table_of_a_64_token_scheme_covers_every_block_once_whatever_the_cells_choose(grid, cand):
+    from paper_2608_03335_b200 import binding
+    # the attention stage pairs 64-token query blocks inside 2 x 2 x 2 cells of the block grid, along an axis chosen per
+    # cell: for every axis the tiles of a cell must hold each of its blocks exactly once, partners one step along that
+    # axis, and the tile count may not depend on the choice
+    plan = binding.Plan(1, 1, grid, 0, (cand,), "sparsity", 0.5)
+    g = plan.geometry(0)
+    nbt, nbh, nbw = g["nbt"], g["nbh"], g["nbw"]
+    tile_cell, pairs = plan.pair_table(0)
+    assert tile_cell.shape[0] == pairs.shape[0]
+    assert (tile_cell[1:] >= tile_cell[:-1]).all(), "the tiles of a cell are consecutive"
+    nct, nch, ncw = (nbt + 1) // 2, (nbh + 1) // 2, (nbw + 1) // 2
+    assert int(tile_cell.max()) + 1 == nct * nch * ncw
+    stride = (nbh * nbw, nbw, 1)
+    for a in range(3):
+        seen = torch.zeros(g["NBv"], dtype=torch.int64)
+        for t in range(pairs.shape[0]):
+            e = int(pairs[t, a])
+            qb0, qb1 = e & 0xffff, e >> 16
+            cell = int(tile_cell[t])
+            blocks = [qb0] if qb1 == 0xffff else [qb0, qb1]
+            if qb1 != 0xffff:
+                assert qb1 - qb0 in stride, "partners are neighbours along one axis"
+            for b in blocks:
+                it, ih, iw = b // (nbh * nbw), (b // nbw) % nbh, b % nbw
+                assert ((it // 2) * nch + ih // 2) * ncw + iw // 2 == cell, "both blocks lie in the tile's cell"
+                seen[b] += 1
+        assert (seen == 1).all(), f"axis {a}: every video block in exactly one tile"
