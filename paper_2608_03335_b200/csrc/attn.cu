@@ -582,7 +582,7 @@ k_attn(const __grid_constant__ AttnMaps maps, const __grid_constant__ Shape sh, 
             if (!__all_sync(FULL, ptx::mbar_wait(&ctl.pv_done, hp & 1, &ctl.abort, WAIT_NS))) { site = 11; break; }
             ptx::tc_fence_after();
             const float alpha = grow ? ptx::ex2((m - m_new) * scale_log2) : 1.f;
-#pragma unroll
+#pragma unroll 1                                  // rare, and the unit loop has to stay short for the instruction cache
             for (int ch = 0; ch < 4; ++ch) {
               uint32_t o[32];
               ptx::tmem_ld32(tmem_O + lane_base + ch * 32, o);
