@@ -133,7 +133,7 @@ __device__ __forceinline__ void store_o_block(const uint8_t* src, const CandMaps
     ptx::tma_store_3d(&tm.o, src, 0, row, bh);
     ptx::tma_store_3d(&tm.o, src + SUB_BYTES, 64, row, bh);
   } else {
-    const int iw = blk % g.nbw, ih = (blk / g.nbw) % g.nbh, it = blk / (g.nbw * g.nbh);   // once per item, in a softmax thread: the divisions stay (the multiply form moved the hot loop's registers and cost 14 %)
+    const int iw = blk % g.nbw, ih = (blk / g.nbw) % g.nbh, it = blk / (g.nbw * g.nbh);   // once per item: the divisions stay (nothing to win here; the 14 % once measured against the multiply form was code placement, see ATT_CODE_PAD)
     ptx::tma_store_5d(&vm.o, src, 0, iw * g.bw, ih * g.bh, it * g.bt, bh);
     ptx::tma_store_5d(&vm.o, src + SUB_BYTES, 64, iw * g.bw, ih * g.bh, it * g.bt, bh);
   }
